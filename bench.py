@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the aggregation primitive (AP) hot path on B200.
+
+One step = one forward AP (mean) + one backward AP (mean) over a synthetic graph shaped like the
+paper's Reddit workload (232,965 vertices, 114,615,892 directed edges, 602 features), through
+the C ABI of libdgagg.  The graph ingest and the CSR->CSC build run once per graph (as in
+training, where the graph is static over epochs); they are timed separately and reported under
+"ingest".  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                  [--workload NAME] [--scale S] [--feat F] [--op sum|mean]
+
+N > 1 (under torchrun): the path has no exchange step and is not sharded, so every rank runs
+an independent replica of the same workload; the value is the units all ranks processed over
+the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "ap_fwd_bwd_edge_feat_per_s"
+UNIT = "edge*feat/s"
+NORTH_STAR_HBM_GBS = 8000.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="reddit_like")
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--feat", type=int, default=0, help="feature width (0 = the workload's)")
+    ap.add_argument("--op", default=None, choices=[None, "sum", "mean"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-seconds", type=float, default=15.0,
+                    help="target CPU time of the oracle sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--set", action="append", default=[],
+                    help="library knob name=value (heavy_threshold, slice_features, rows_per_block)")
+    return ap.parse_args()
+
+
+def default_op(workload):
+    return {"reddit_like": "mean", "products_like": "mean"}.get(workload, "sum")
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def compulsory_bytes(n, nnz, F, weighted, n_ref, inv_deg_gather):
+    """Bytes one AP call must move once: pointers, indices, weights, the referenced rows of the
+    input matrix read once, the output written once (+ the 1/deg vector for the mean backward)."""
+    b = (n + 1) * 8 + nnz * 4 + (nnz * 4 if weighted else 0) + n_ref * F * 4 + n * F * 4
+    if inv_deg_gather:
+        b += n * 4
+    return b
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 8:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def oracle_sample(sg_host, H, G, op_code, n_rows, seed=0):
+    """Runs the oracle (forward over sampled rows, backward over sampled columns) and returns
+    (edge*feat processed, seconds)."""
+    import numpy as np
+    import oracle
+    rowptr, colidx, w, colptr, rowidx_T, w_T = sg_host
+    n = rowptr.shape[0] - 1
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(n, size=min(n_rows, n), replace=False))
+    F = H.shape[1]
+    work = int((rowptr[rows + 1] - rowptr[rows]).sum() + (colptr[rows + 1] - colptr[rows]).sum()) * F
+    t0 = time.perf_counter()
+    oracle.ap_forward(rowptr, colidx, w, H, op_code, rows=rows)
+    oracle.ap_backward(rowptr, colptr, rowidx_T, w_T, G, op_code, cols=rows)
+    return work, time.perf_counter() - t0
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle, as it stands, on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    import oracle
+    from paper_2104_06700_b200 import synth
+    op = args.op or default_op(args.workload)
+    op_code = oracle.OP_MEAN if op == "mean" else oracle.OP_SUM
+    import torch
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    sg = synth.make(args.workload, device=dev, scale=args.scale)
+    F = args.feat or sg.F
+    rowptr, colidx = sg.rowptr.cpu().numpy(), sg.colidx.cpu().numpy()
+    w = None if sg.edge_w is None else sg.edge_w.cpu().numpy()
+    colptr, rowidx_T, w_T, _ = oracle.transpose(rowptr, colidx, w)
+    H = synth.features(sg.n, F, 100, "cpu").numpy()
+    G = synth.features(sg.n, F, 101, "cpu").numpy()
+    host = (rowptr, colidx, w, colptr, rowidx_T, w_T)
+    # size the sample so that all steps together take about two minutes at most
+    work, sec = oracle_sample(host, H, G, op_code, 64)
+    per_row = sec / 64
+    budget = min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup))
+    n_rows = int(max(64, min(sg.n, budget / max(per_row, 1e-9))))
+    for i in range(args.warmup):
+        oracle_sample(host, H, G, op_code, n_rows, seed=i)
+    tot_work, tot_sec = 0, 0.0
+    for i in range(args.steps):
+        wk, sc = oracle_sample(host, H, G, op_code, n_rows, seed=1000 + i)
+        tot_work += wk
+        tot_sec += sc
+    value = tot_work / tot_sec
+    sample = f"{n_rows} sampled destination rows (fwd) and source columns (bwd) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_sec / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
+                   "F": F, "op": op},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2104_06700_b200 import binding, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the aggregation kernels have no fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    op = args.op or default_op(args.workload)
+    op_code = binding.DG_OP_MEAN if op == "mean" else binding.DG_OP_SUM
+
+    # ---------------------------------------------------------------- inputs (seeded, synthetic)
+    sg = synth.make(args.workload, device=dev, scale=args.scale)
+    F = args.feat or sg.F
+    H = synth.features(sg.n, F, 100, dev)
+    G = synth.features(sg.n, F, 101, dev)
+    out = torch.empty_like(H)
+    dH = torch.empty_like(H)
+    weighted = sg.edge_w is not None
+    n_ref = int((torch.bincount(sg.colidx.long(), minlength=sg.n) > 0).sum())
+    n_rows_nonempty = int(((sg.rowptr[1:] - sg.rowptr[:-1]) > 0).sum())
+
+    # ---------------------------------------------------------------- ingest (once per graph)
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+    torch.cuda.synchronize()
+    create_ms = 1e3 * (time.perf_counter() - t0)
+    for name_value in args.set:
+        k, v = name_value.split("=")
+        g.dg_graph_set_param(k, int(v))
+    need_csc, need_scratch = g.dg_graph_transpose_workspace()
+    csc = torch.empty(need_csc, dtype=torch.uint8, device=dev)
+    scratch = torch.empty(need_scratch, dtype=torch.uint8, device=dev)
+    g.dg_graph_transpose(csc, scratch)          # warm-up
+    torch.cuda.synchronize()
+    e0, e1 = ev(), ev()
+    e0.record(stream)
+    g.dg_graph_transpose(csc, scratch)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    transpose_ms = e0.elapsed_time(e1)
+    del scratch
+
+    # ---------------------------------------------------------------- device-resident timing
+    def step():
+        g.dg_aggregate_fwd(H, op_code, out=out)
+        g.dg_aggregate_bwd(G, op_code, dH=dH)
+
+    for _ in range(max(3, args.warmup)):
+        step()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    launches0 = binding.dg_kernel_launch_count()
+    marks = [ev() for _ in range(2 * args.steps + 1)]
+    torch.cuda.synchronize()
+    marks[0].record(stream)
+    for i in range(args.steps):
+        g.dg_aggregate_fwd(H, op_code, out=out)
+        marks[2 * i + 1].record(stream)
+        g.dg_aggregate_bwd(G, op_code, dH=dH)
+        marks[2 * i + 2].record(stream)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    launches = binding.dg_kernel_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = marks[0].elapsed_time(marks[-1])
+    fwd_ms = sum(marks[2 * i].elapsed_time(marks[2 * i + 1]) for i in range(args.steps)) / args.steps
+    bwd_ms = sum(marks[2 * i + 1].elapsed_time(marks[2 * i + 2]) for i in range(args.steps)) / args.steps
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    units_per_step = 2 * sg.nnz * F                 # forward + backward edge*feature products
+    value = world * units_per_step / (ms_per_step * 1e-3)
+
+    # ---------------------------------------------------------------- roofline of the dominant kernel
+    peak, peak_kind = measured_peaks()
+    b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False)
+    b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_rows_nonempty, op == "mean")
+    dom = "fwd" if fwd_ms >= bwd_ms else "bwd"
+    dom_ms, dom_bytes = (fwd_ms, b_fwd) if dom == "fwd" else (bwd_ms, b_bwd)
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": f"ap_kernel ({dom}: one launch per dg_aggregate_{dom} call)",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "peak_kind": f"of {peak_kind}", "frac_of_north_star_8TBs": achieved / NORTH_STAR_HBM_GBS,
+        "algorithmic_bytes_per_launch": dom_bytes, "ms_per_launch": dom_ms, "traffic": None,
+        "fwd": {"ms": fwd_ms, "bytes": b_fwd, "GBs": b_fwd / fwd_ms / 1e6,
+                "edge_feat_per_s": sg.nnz * F / (fwd_ms * 1e-3)},
+        "bwd": {"ms": bwd_ms, "bytes": b_bwd, "GBs": b_bwd / bwd_ms / 1e6,
+                "edge_feat_per_s": sg.nnz * F / (bwd_ms * 1e-3)},
+        "gather_bytes_per_launch": sg.nnz * F * 4,
+        "gather_GBs": sg.nnz * F * 4 / (dom_ms * 1e-3) / 1e9,
+    }
+
+    # ---------------------------------------------------------------- end to end from host memory
+    e2e = None
+    if args.e2e_steps > 0:
+        Hh = torch.empty((sg.n, F), dtype=torch.float32).pin_memory()
+        Gh = torch.empty((sg.n, F), dtype=torch.float32).pin_memory()
+        Hh.copy_(H); Gh.copy_(G)
+        outh = torch.empty_like(Hh).pin_memory()
+        dHh = torch.empty_like(Hh).pin_memory()
+        ws = torch.empty(g.dg_aggregate_host_workspace(F), dtype=torch.uint8, device=dev)
+        g.dg_aggregate_host(Hh, Gh, op_code, outh, dHh, ws)
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(args.e2e_steps):
+            g.dg_aggregate_host(Hh, Gh, op_code, outh, dHh, ws)
+        b.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms = a.elapsed_time(b)
+        if world > 1:
+            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_ms = float(t.item())
+        e2e_ms /= args.e2e_steps
+        e2e = {"value": world * units_per_step / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": 2 * sg.n * F * 4, "d2h_bytes_per_step": 2 * sg.n * F * 4,
+               "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+               "call": "dg_aggregate_host (pinned host H, dOut in; out, dH back)"}
+        del Hh, Gh, outh, dHh, ws
+
+    # ---------------------------------------------------------------- CPU baseline (rank 0, N=1)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
+        host = (sg.rowptr.cpu().numpy(), sg.colidx.cpu().numpy(),
+                None if sg.edge_w is None else sg.edge_w.cpu().numpy(),
+                colptr.cpu().numpy(), rowidx_T.cpu().numpy(),
+                None if w_T is None else w_T.cpu().numpy())
+        Hn, Gn = H.cpu().numpy(), G.cpu().numpy()
+        o_op = oracle.OP_MEAN if op == "mean" else oracle.OP_SUM
+        wk, sc = oracle_sample(host, Hn, Gn, o_op, 64)
+        n_rows = int(max(64, min(sg.n, args.cpu_seconds / max(sc / 64, 1e-9))))
+        wk, sc = oracle_sample(host, Hn, Gn, o_op, n_rows, seed=1)
+        cpu = {"value": wk / sc, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{n_rows} of {sg.n} destination rows (fwd) and source columns (bwd), "
+                         f"{sc:.1f} s, fp64 accumulation"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
+                       "F": F, "op": op, "weighted": weighted, "step": "fwd AP + bwd AP",
+                       "replicas": world, "l2": "inputs larger than L2 (no flush needed)"
+                       if sg.n * F * 4 > 252e6 else "inputs fit L2: warm-L2 numbers",
+                       "knobs": args.set},
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks,
+            "ingest": {"graph_create_ms": create_ms, "transpose_ms": transpose_ms,
+                       "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3) if transpose_ms else None},
+        }))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,163 @@
+/*
+ * libdgagg -- the aggregation primitive (AP) of full-batch GraphSAGE training on one B200.
+ *
+ * AP is the sparse-times-dense product f_O = A x f_V of Section 2.1 of the paper (Eq. 1 with
+ * the binary operator "multiply by the edge's scalar weight", Eq. 2 with the unary copy, both
+ * with the reducer "sum" of Table 1), computed in the pull form of Algorithm 1: the CSR row of
+ * a destination vertex v lists the source vertices u that have an edge u -> v (Section 3.1).
+ * "mean" divides the sum by the in-degree of v, the normalisation of Section 5.1 (Models and
+ * Parameters).  The backward pass dH = A^T x dOut and the CSR -> CSC build it needs are not
+ * written in the paper; they are the adjoint of the forward pass and a stable counting sort.
+ *
+ * Conventions for every entry point
+ *   - plain C ABI, no exceptions cross it; every call returns a dg_status_t, and
+ *     dg_last_error() gives a message for the last failure on the calling thread;
+ *   - "device" pointers are CUDA device memory of the current device, "host" pointers are
+ *     ordinary process memory; the library never takes ownership of a caller's buffer;
+ *   - `stream` is a CUDA stream handle (cudaStream_t / CUstream passed as void*); NULL is the
+ *     legacy default stream.  Calls that take a stream only enqueue work on it;
+ *   - feature matrices are dense, row-major, fp32, leading dimension F;
+ *   - rowptr/colptr are int64, vertex ids are int32 (n < 2^31), nnz < 2^31;
+ *   - no call aborts, traps or waits without bound on the device.
+ */
+#ifndef DG_H_
+#define DG_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DG_OK = 0,
+  DG_ERR_INVALID_ARG = 1,     /* null pointer, negative size, aliasing, bad enum            */
+  DG_ERR_UNSUPPORTED = 2,     /* a size beyond the limits stated above                      */
+  DG_ERR_CUDA = 3,            /* a CUDA runtime call failed; dg_last_error() has its text   */
+  DG_ERR_NOT_TRANSPOSED = 4,  /* backward pass or CSC query before dg_graph_transpose       */
+  DG_ERR_WORKSPACE = 5,       /* csc_storage or scratch smaller than the workspace query    */
+  DG_ERR_INVALID_GRAPH = 6    /* dg_graph_validate found a malformed CSR                    */
+} dg_status_t;
+
+/* Reducer of Table 1 ("sum"), and the sum divided by the in-degree (Section 5.1). */
+typedef enum { DG_OP_SUM = 0, DG_OP_MEAN = 1 } dg_op_t;
+
+typedef struct dg_graph* dg_graph_t;
+
+/*
+ * Graph ingest: records the CSR of A (Section 3.1: rows = destination vertices, column
+ * indices = source vertices, any order inside a row, duplicates and self-loops allowed).
+ *   n       number of vertices, 0 <= n < 2^31
+ *   nnz     number of directed edges, 0 <= nnz < 2^31
+ *   rowptr  device, n+1 entries, rowptr[0] = 0, non-decreasing, rowptr[n] = nnz
+ *   colidx  device, nnz entries in [0, n)
+ *   edge_w  device, nnz fp32 scalars (the edge feature of Eq. 1 reduced to one value per
+ *           edge and broadcast over the F features), or NULL for the unary copy of Eq. 2
+ * The handle BORROWS the three arrays: they must stay valid and unchanged until
+ * dg_graph_destroy.  The call allocates a few small device arrays that it owns (1/in-degree
+ * per vertex, the lists of heavy rows) and synchronises the device once.
+ * The arrays are trusted; dg_graph_validate checks them.
+ */
+dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
+                            const int32_t* colidx, const float* edge_w, dg_graph_t* out_graph);
+
+/* Frees what dg_graph_create allocated.  The borrowed CSR and the caller's CSC storage are
+ * not touched.  NULL is accepted. */
+dg_status_t dg_graph_destroy(dg_graph_t g);
+
+/* Synchronous check of the borrowed CSR on `stream`: rowptr[0] = 0, rowptr non-decreasing,
+ * rowptr[n] = nnz, every colidx in [0, n).  Returns DG_ERR_INVALID_GRAPH if not. */
+dg_status_t dg_graph_validate(dg_graph_t g, void* stream);
+
+/* Sizes in bytes of the two device buffers dg_graph_transpose needs for this graph. */
+dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t* scratch_bytes);
+
+/*
+ * CSR -> CSC on the GPU (the paper works on the CSR only and leaves this step implicit).
+ * The result is the stable counting sort of the edge positions k = 0..nnz-1 by colidx[k]:
+ *   colptr[u]   number of edges with source < u (int64, n+1 entries)
+ *   perm[q]     CSR position of the q-th edge in (source, position) order (int32)
+ *   rowidx_T[q] destination vertex of edge perm[q] (int32)
+ *   w_T[q]      edge_w[perm[q]], copied bit for bit (absent when the graph is unweighted)
+ * There is exactly one correct result; it is integer work and bit-exact.
+ *   csc_storage  device, 256-byte aligned, >= csc_bytes; holds the four arrays, is borrowed
+ *                by the handle until destroy (or the next transpose) and is what
+ *                dg_graph_get_csc points into
+ *   scratch      device, 256-byte aligned, >= scratch_bytes; free for reuse once the work
+ *                enqueued on `stream` has finished
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes,
+                               void* scratch, size_t scratch_bytes, void* stream);
+
+/* Device pointers to the CSC arrays inside csc_storage (any output pointer may be NULL).
+ * *w_T is set to NULL for an unweighted graph. */
+dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t** rowidx_T,
+                             const float** w_T, const int32_t** perm);
+
+/*
+ * Forward AP (Algorithm 1 with the operators above):
+ *   out[v][j] = s_v * sum over the CSR row of v of  w_k * H[colidx[k]][j],   0 <= j < F
+ * w_k = edge_w[k] (1 if unweighted); s_v = 1 for DG_OP_SUM, 1/deg(v) for DG_OP_MEAN with
+ * deg(v) = rowptr[v+1]-rowptr[v]; a vertex without in-edges gets zeros (the output of
+ * Algorithm 1 starts at zero).
+ *   H    device, n x F fp32 row-major, read only
+ *   out  device, n x F fp32 row-major, OVERWRITTEN (no need to clear it); must not overlap H
+ * fp32 accumulation in a fixed order: the same call on the same data gives the same bits.
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op, float* out,
+                             void* stream);
+
+/*
+ * Backward AP, the adjoint of dg_aggregate_fwd with the same (F, op):
+ *   dH[u][j] = sum over the CSC segment of u of  w_T[q] * s_{v_q} * dOut[v_q][j],
+ *   v_q = rowidx_T[q]
+ * (the mean's 1/deg belongs to the destination vertex v_q).  Gathers over the CSC built by
+ * dg_graph_transpose, without atomics, in a fixed order.  dH is OVERWRITTEN and must not
+ * overlap dOut.  Returns DG_ERR_NOT_TRANSPOSED before dg_graph_transpose.
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t op, float* dH,
+                             void* stream);
+
+/*
+ * Forward and backward AP with the feature matrices in HOST memory (pinned memory makes the
+ * copies asynchronous and faster; pageable memory works).  Equivalent to copying H_host and
+ * dOut_host into device_ws, calling dg_aggregate_fwd and dg_aggregate_bwd, and copying the
+ * results into out_host and dH_host, all on `stream`.  dOut_host/dH_host may both be NULL to
+ * run the forward pass only.
+ *   device_ws  device, 256-byte aligned, >= dg_aggregate_host_workspace(g, F) bytes
+ * Asynchronous on `stream` when the host buffers are pinned; the host results are complete
+ * once the stream has been synchronised.
+ */
+size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F);
+dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dOut_host,
+                              int32_t F, dg_op_t op, float* out_host, float* dH_host,
+                              void* device_ws, size_t device_ws_bytes, void* stream);
+
+/*
+ * Tuning knobs (defaults come from the device's L2 size and SM count):
+ *   "heavy_threshold"  rows longer than this are summed by a whole thread block
+ *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
+ *   "rows_per_block"   destination rows per thread block in the light-row kernel
+ * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.
+ */
+dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);
+dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value);
+
+/* Number of kernels the library has launched from this process (all handles, all threads). */
+int64_t dg_kernel_launch_count(void);
+
+/* Message of the last failure on this thread ("" if none).  Valid until the next failing call
+ * on the same thread. */
+const char* dg_last_error(void);
+
+/* "libdgagg <version> sm_100a". */
+const char* dg_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DG_H_ */

@@ -1,0 +1,290 @@
+// Aggregation kernels: out[r] = rs_r * sum_k s_k * X[idx[k]] over one segment of a CSR (forward)
+// or CSC (backward) structure.  This is the pull loop of Algorithm 1 of the paper; the register
+// accumulation with one store per row follows the idea of Algorithm 3, and the split of the
+// feature dimension into slices that keep the gathered matrix L2-resident plays the role that
+// source blocking (Algorithm 2) plays on a CPU cache.
+//
+// Work decomposition
+//   light segments (length <= heavy_threshold): one warp per segment.  Lanes are spread along
+//     the feature dimension with 16-, 8- or 4-byte vector loads.  When a row slice needs fewer
+//     than 32 vectors the warp is cut into groups of G lanes and the groups take different
+//     edges of the same segment; their partial sums are combined by a fixed shuffle tree.
+//   heavy segments: one thread block per segment (the first blocks of the same launch loop over
+//     the heavy list); the 8 warps take interleaved batches of 32 edges and combine in shared
+//     memory in warp order.
+// Every output element is produced by one thread in an order fixed by the launch shape, so the
+// result is deterministic and needs no atomics in either direction.
+#include "dg_internal.cuh"
+
+namespace dg {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kBlock = kWarpsPerBlock * 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+template <int VEC> struct Vec;
+template <> struct Vec<1> { using T = float; };
+template <> struct Vec<2> { using T = float2; };
+template <> struct Vec<4> { using T = float4; };
+
+__device__ __forceinline__ float ldg_vec(const float* p, float) { return __ldg(p); }
+__device__ __forceinline__ float2 ldg_vec(const float* p, float2) {
+  return __ldg(reinterpret_cast<const float2*>(p));
+}
+__device__ __forceinline__ float4 ldg_vec(const float* p, float4) {
+  return __ldg(reinterpret_cast<const float4*>(p));
+}
+__device__ __forceinline__ void zero(float& a) { a = 0.f; }
+__device__ __forceinline__ void zero(float2& a) { a.x = a.y = 0.f; }
+__device__ __forceinline__ void zero(float4& a) { a.x = a.y = a.z = a.w = 0.f; }
+__device__ __forceinline__ void add(float& a, const float& v) { a += v; }
+__device__ __forceinline__ void add(float2& a, const float2& v) { a.x += v.x; a.y += v.y; }
+__device__ __forceinline__ void add(float4& a, const float4& v) {
+  a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+}
+__device__ __forceinline__ void fma(float& a, float s, const float& v) { a = fmaf(s, v, a); }
+__device__ __forceinline__ void fma(float2& a, float s, const float2& v) {
+  a.x = fmaf(s, v.x, a.x); a.y = fmaf(s, v.y, a.y);
+}
+__device__ __forceinline__ void fma(float4& a, float s, const float4& v) {
+  a.x = fmaf(s, v.x, a.x); a.y = fmaf(s, v.y, a.y);
+  a.z = fmaf(s, v.z, a.z); a.w = fmaf(s, v.w, a.w);
+}
+__device__ __forceinline__ void scale(float& a, float s) { a *= s; }
+__device__ __forceinline__ void scale(float2& a, float s) { a.x *= s; a.y *= s; }
+__device__ __forceinline__ void scale(float4& a, float s) { a.x *= s; a.y *= s; a.z *= s; a.w *= s; }
+__device__ __forceinline__ float shfl_xor(float a, int m) { return __shfl_xor_sync(kFull, a, m); }
+__device__ __forceinline__ float2 shfl_xor(float2 a, int m) {
+  return make_float2(__shfl_xor_sync(kFull, a.x, m), __shfl_xor_sync(kFull, a.y, m));
+}
+__device__ __forceinline__ float4 shfl_xor(float4 a, int m) {
+  return make_float4(__shfl_xor_sync(kFull, a.x, m), __shfl_xor_sync(kFull, a.y, m),
+                     __shfl_xor_sync(kFull, a.z, m), __shfl_xor_sync(kFull, a.w, m));
+}
+__device__ __forceinline__ void stcs_vec(float* p, float v) { __stcs(p, v); }
+__device__ __forceinline__ void stcs_vec(float* p, float2 v) { __stcs(reinterpret_cast<float2*>(p), v); }
+__device__ __forceinline__ void stcs_vec(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+__device__ __forceinline__ void st_smem(float* p, float v) { p[0] = v; }
+__device__ __forceinline__ void st_smem(float* p, float2 v) { p[0] = v.x; p[1] = v.y; }
+__device__ __forceinline__ void st_smem(float* p, float4 v) {
+  p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
+}
+
+// Loads the neighbour id and the per-edge factor of edge k (k < hi), else a neutral pair.
+template <bool SCALED>
+__device__ __forceinline__ void load_edge(const ApArgs& a, int64_t k, int64_t hi, int32_t& u,
+                                          float& s) {
+  u = 0;
+  s = 0.f;
+  if (k < hi) {
+    u = __ldcs(a.idx + k);
+    if (SCALED) {
+      s = a.w ? __ldcs(a.w + k) : 1.f;
+      if (a.node_scale) s *= __ldg(a.node_scale + u);
+    }
+  }
+}
+
+// Sums the edges of [lo, hi) that fall into batches first, first+step, ... (32 edges each) into
+// acc.  Within a batch, lane group `grp` takes edges grp, grp+NG, ...; U edges are in flight
+// per group.
+template <int VEC, int G, int CPL, bool SCALED>
+__device__ __forceinline__ void accumulate(const ApArgs& a, int64_t lo, int64_t hi, int first,
+                                           int step, int f0, int fend,
+                                           typename Vec<VEC>::T (&acc)[CPL]) {
+  using V = typename Vec<VEC>::T;
+  constexpr int NG = 32 / G;
+  constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : 2);
+  constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;
+  const int lane = threadIdx.x & 31;
+  const int grp = lane / G;
+  const int c0 = lane % G;
+
+  int foff[CPL];
+  bool fok[CPL];
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) {
+    foff[c] = f0 + (c0 + c * G) * VEC;
+    fok[c] = foff[c] < fend;
+  }
+
+  int64_t base = lo + (int64_t)first * 32;
+  int32_t my_u, nx_u;
+  float my_s, nx_s;
+  if (base < hi) load_edge<SCALED>(a, base + lane, hi, nx_u, nx_s);
+  for (; base < hi; base += (int64_t)step * 32) {
+    my_u = nx_u;
+    my_s = nx_s;
+    const int64_t nbase = base + (int64_t)step * 32;
+    if (nbase < hi) load_edge<SCALED>(a, nbase + lane, hi, nx_u, nx_s);
+    const int cnt = (hi - base) < 32 ? (int)(hi - base) : 32;
+    for (int e0 = 0; e0 < cnt; e0 += U * NG) {
+      V v[U][CPL];
+      float s[U];
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int e = e0 + j * NG + grp;
+        const bool ok = e < cnt;
+        const int32_t u = __shfl_sync(kFull, my_u, e & 31);
+        s[j] = SCALED ? __shfl_sync(kFull, my_s, e & 31) : 1.f;
+        const float* row = a.X + (size_t)u * (size_t)a.F;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          if (ok && fok[c]) v[j][c] = ldg_vec(row + foff[c], V());
+          else zero(v[j][c]);
+        }
+        if (!ok) s[j] = 0.f;
+      }
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          if (SCALED) fma(acc[c], s[j], v[j][c]);
+          else add(acc[c], v[j][c]);
+        }
+      }
+    }
+  }
+  // combine the lane groups (fixed tree)
+#pragma unroll
+  for (int off = G; off < 32; off <<= 1) {
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) add(acc[c], shfl_xor(acc[c], off));
+  }
+}
+
+// One launch does both roles: blocks [0, heavy_blocks) walk the heavy list (they are scheduled
+// first, so the long segments start early), the remaining blocks take rows_per_block consecutive
+// light segments each.
+template <int VEC, int G, int CPL, bool SCALED>
+__global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
+  using V = typename Vec<VEC>::T;
+  __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int f0 = blockIdx.y * a.slice_f;
+  const int fend = min(a.F, f0 + a.slice_f);
+  const int c0 = lane % G;
+
+  if ((int)blockIdx.x >= heavy_blocks) {
+    const int64_t row0 = (int64_t)(blockIdx.x - heavy_blocks) * a.rows_per_block;
+    const int64_t row1 = min(a.n, row0 + a.rows_per_block);
+    for (int64_t r = row0 + warp; r < row1; r += kWarpsPerBlock) {
+      const int64_t lo = __ldg(a.ptr + r), hi = __ldg(a.ptr + r + 1);
+      const int64_t len = hi - lo;
+      if (len > a.heavy_threshold) continue;  // a heavy block writes this row
+      V acc[CPL];
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) zero(acc[c]);
+      accumulate<VEC, G, CPL, SCALED>(a, lo, hi, 0, 1, f0, fend, acc);
+      if (lane < G) {
+        const float rs = (a.mean_rows && len > 0) ? 1.0f / (float)len : 1.0f;
+        float* orow = a.Y + (size_t)r * (size_t)a.F;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) {
+          const int f = f0 + (c0 + c * G) * VEC;
+          if (f < fend) {
+            if (a.mean_rows) scale(acc[c], rs);
+            stcs_vec(orow + f, acc[c]);
+          }
+        }
+      }
+    }
+    return;
+  }
+
+  const int width = fend - f0;
+  const int count = min(*a.heavy_count, a.heavy_cap);
+  for (int i = blockIdx.x; i < count; i += heavy_blocks) {
+    const int64_t r = a.heavy_list[i];
+    const int64_t lo = __ldg(a.ptr + r), hi = __ldg(a.ptr + r + 1);
+    V acc[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) zero(acc[c]);
+    accumulate<VEC, G, CPL, SCALED>(a, lo, hi, warp, kWarpsPerBlock, f0, fend, acc);
+    if (lane < G) {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        const int fl = (c0 + c * G) * VEC;
+        if (fl < width) st_smem(&part[warp][fl], acc[c]);
+      }
+    }
+    __syncthreads();
+    const float rs = a.mean_rows ? 1.0f / (float)(hi - lo) : 1.0f;
+    float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
+    for (int f = threadIdx.x; f < width; f += kBlock) {
+      float t = part[0][f];
+#pragma unroll
+      for (int w = 1; w < kWarpsPerBlock; ++w) t += part[w][f];
+      __stcs(orow + f, a.mean_rows ? t * rs : t);
+    }
+    __syncthreads();
+  }
+}
+
+template <int VEC, int G, int CPL, bool SCALED>
+dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
+  if (a.n == 0) return DG_OK;
+  const int heavy_blocks = g->sm_count * 2;
+  const int64_t blocks = heavy_blocks + (a.n + a.rows_per_block - 1) / a.rows_per_block;
+  dim3 grid((unsigned)blocks, (unsigned)slices);
+  ap_kernel<VEC, G, CPL, SCALED><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
+}
+
+template <int VEC, bool SCALED>
+dg_status_t dispatch_shape(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
+  const int chunks = (a.slice_f < a.F ? a.slice_f : a.F) / VEC;  // vectors per row slice
+  if (chunks <= 2) return launch_pair<VEC, 2, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 4) return launch_pair<VEC, 4, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 8) return launch_pair<VEC, 8, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 16) return launch_pair<VEC, 16, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 32) return launch_pair<VEC, 32, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 64) return launch_pair<VEC, 32, 2, SCALED>(g, a, slices, s);
+  return launch_pair<VEC, 32, 4, SCALED>(g, a, slices, s);
+}
+
+}  // namespace
+
+// Widest vector both matrices allow, then the slice width: at most 128 vectors per row slice
+// (4 per lane), narrowed until one slice of X fits the L2 budget so that repeated gathers of a
+// source row are served from L2 instead of HBM.
+dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, cudaStream_t s) {
+  ApArgs a = a0;
+  const uintptr_t px = (uintptr_t)a.X, py = (uintptr_t)a.Y;
+  int vec = 1;
+  if (a.F % 4 == 0 && px % 16 == 0 && py % 16 == 0) vec = 4;
+  else if (a.F % 2 == 0 && px % 8 == 0 && py % 8 == 0) vec = 2;
+
+  int64_t slice = g->slice_features;
+  if (slice <= 0) {
+    slice = a.F;
+    const double budget = 0.4 * (double)g->l2_bytes;
+    if ((double)a.n * a.F * 4.0 > budget) {
+      slice = (int64_t)(budget / ((double)a.n * 4.0));
+      if (slice < 32) slice = a.F;  // a slice under 128 bytes per row is not worth a pass
+    }
+  }
+  const int64_t cap = 128LL * vec;
+  if (slice > cap) slice = cap;
+  if (slice > a.F) slice = a.F;
+  slice = (slice / vec) * vec;
+  if (slice < vec) slice = vec;
+  // even out the slices: same count, smallest width that covers F
+  const int64_t nsl = (a.F + slice - 1) / slice;
+  int64_t even = (a.F + nsl - 1) / nsl;
+  even = ((even + vec - 1) / vec) * vec;
+  if (even <= slice) slice = even;
+  a.slice_f = (int32_t)slice;
+  const int slices = (int)((a.F + slice - 1) / slice);
+  const bool scaled = a.w != nullptr || a.node_scale != nullptr;
+
+  if (vec == 4) return scaled ? dispatch_shape<4, true>(g, a, slices, s) : dispatch_shape<4, false>(g, a, slices, s);
+  if (vec == 2) return scaled ? dispatch_shape<2, true>(g, a, slices, s) : dispatch_shape<2, false>(g, a, slices, s);
+  return scaled ? dispatch_shape<1, true>(g, a, slices, s) : dispatch_shape<1, false>(g, a, slices, s);
+}
+
+}  // namespace dg

@@ -1,0 +1,304 @@
+// The C ABI of libdgagg: argument checks, handle bookkeeping and kernel dispatch.
+// Declarations and the meaning of every argument are in include/dg.h.
+#include <string.h>
+
+#include <new>
+
+#include "dg_internal.cuh"
+
+namespace dg {
+
+static thread_local std::string g_last_error;
+static std::atomic<int64_t> g_launches{0};
+
+void set_error(const std::string& msg) { g_last_error = msg; }
+
+dg_status_t cuda_fail(cudaError_t e, const char* what) {
+  g_last_error = std::string(what) + ": " + cudaGetErrorString(e);
+  return DG_ERR_CUDA;
+}
+
+void count_launches(int64_t k) { g_launches.fetch_add(k, std::memory_order_relaxed); }
+
+static dg_status_t invalid(const char* msg) {
+  set_error(msg);
+  return DG_ERR_INVALID_ARG;
+}
+
+static bool overlaps(const void* a, const void* b, size_t bytes) {
+  const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
+  return x < y + bytes && y < x + bytes;
+}
+
+static dg_status_t free_owned(Graph* g) {
+  if (g->inv_deg) cudaFree(g->inv_deg);
+  if (g->heavy_rows) cudaFree(g->heavy_rows);
+  if (g->heavy_cols) cudaFree(g->heavy_cols);
+  if (g->counters) cudaFree(g->counters);
+  g->inv_deg = nullptr;
+  g->heavy_rows = g->heavy_cols = g->counters = nullptr;
+  return DG_OK;
+}
+
+// (Re)builds the heavy lists for the current threshold; called at create, after a transpose
+// and after the threshold changes.
+static dg_status_t refresh_heavy(Graph* g, bool csr, bool csc, cudaStream_t s) {
+  if (csr)
+    if (dg_status_t st = build_heavy_list(g->rowptr, g->n, g->heavy_threshold, g->heavy_rows,
+                                          g->heavy_cap, g->counters + 0, s))
+      return st;
+  if (csc && g->transposed)
+    if (dg_status_t st = build_heavy_list(g->colptr, g->n, g->heavy_threshold, g->heavy_cols,
+                                          g->heavy_cap, g->counters + 1, s))
+      return st;
+  return DG_OK;
+}
+
+static dg_status_t check_features(const Graph* g, const float* in, float* out, int32_t F,
+                                  dg_op_t op) {
+  if (!g) return invalid("graph handle is NULL");
+  if (F < 1) return invalid("F must be >= 1");
+  if (op != DG_OP_SUM && op != DG_OP_MEAN) return invalid("op must be DG_OP_SUM or DG_OP_MEAN");
+  if (g->n > 0) {
+    if (!in || !out) return invalid("feature matrix pointer is NULL");
+    if (overlaps(in, out, (size_t)g->n * (size_t)F * sizeof(float)))
+      return invalid("input and output feature matrices overlap");
+  }
+  return DG_OK;
+}
+
+}  // namespace dg
+
+using namespace dg;
+
+extern "C" {
+
+dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
+                            const int32_t* colidx, const float* edge_w, dg_graph_t* out_graph) {
+  if (!out_graph) return invalid("out_graph is NULL");
+  *out_graph = nullptr;
+  if (n < 0 || nnz < 0) return invalid("n and nnz must be >= 0");
+  if (n >= ((int64_t)1 << 31) || nnz >= ((int64_t)1 << 31)) {
+    set_error("n and nnz must be below 2^31");
+    return DG_ERR_UNSUPPORTED;
+  }
+  if (!rowptr) return invalid("rowptr is NULL");
+  if (nnz > 0 && !colidx) return invalid("colidx is NULL");
+  if (nnz > 0 && n == 0) return invalid("edges without vertices");
+
+  Graph* g = new (std::nothrow) Graph();
+  if (!g) return invalid("out of host memory");
+  g->n = n;
+  g->nnz = nnz;
+  g->rowptr = rowptr;
+  g->colidx = colidx;
+  g->edge_w = edge_w;
+  cudaError_t e = cudaGetDevice(&g->device);
+  cudaDeviceProp prop;
+  if (e == cudaSuccess) e = cudaGetDeviceProperties(&prop, g->device);
+  if (e != cudaSuccess) { delete g; return cuda_fail(e, "cudaGetDeviceProperties"); }
+  g->sm_count = prop.multiProcessorCount;
+  g->l2_bytes = (size_t)prop.l2CacheSize;
+  g->heavy_cap = nnz / 64 + 1;  // enough for any threshold >= 64
+  if (g->heavy_cap > n) g->heavy_cap = n > 0 ? n : 1;
+
+  e = cudaMalloc(&g->inv_deg, (size_t)(n > 0 ? n : 1) * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_rows, (size_t)g->heavy_cap * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)g->heavy_cap * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&g->counters, 4 * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(g->counters, 0, 4 * sizeof(int32_t));
+  if (e != cudaSuccess) { free_owned(g); delete g; return cuda_fail(e, "cudaMalloc (graph metadata)"); }
+
+  dg_status_t st = build_degree_info(g, 0);
+  if (st == DG_OK) st = refresh_heavy(g, true, false, 0);
+  if (st == DG_OK) {
+    e = cudaStreamSynchronize(0);
+    if (e != cudaSuccess) st = cuda_fail(e, "cudaStreamSynchronize (graph create)");
+  }
+  if (st != DG_OK) { free_owned(g); delete g; return st; }
+  *out_graph = g;
+  return DG_OK;
+}
+
+dg_status_t dg_graph_destroy(dg_graph_t g) {
+  if (!g) return DG_OK;
+  free_owned(g);
+  delete g;
+  return DG_OK;
+}
+
+dg_status_t dg_graph_validate(dg_graph_t g, void* stream) {
+  if (!g) return invalid("graph handle is NULL");
+  int flags = 0;
+  if (dg_status_t st = validate_csr(g, (cudaStream_t)stream, &flags)) return st;
+  if (flags) {
+    std::string m = "malformed CSR:";
+    if (flags & 1) m += " rowptr[0] != 0;";
+    if (flags & 2) m += " rowptr decreases;";
+    if (flags & 4) m += " rowptr[n] != nnz;";
+    if (flags & 8) m += " colidx outside [0, n);";
+    set_error(m);
+    return DG_ERR_INVALID_GRAPH;
+  }
+  return DG_OK;
+}
+
+dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t* scratch_bytes) {
+  if (!g) return invalid("graph handle is NULL");
+  if (!csc_bytes || !scratch_bytes) return invalid("size output is NULL");
+  transpose_sizes(g->n, g->nnz, g->edge_w != nullptr, csc_bytes, scratch_bytes);
+  return DG_OK;
+}
+
+dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes, void* scratch,
+                               size_t scratch_bytes, void* stream) {
+  if (!g) return invalid("graph handle is NULL");
+  if (!csc_storage || !scratch) return invalid("csc_storage or scratch is NULL");
+  if (((uintptr_t)csc_storage | (uintptr_t)scratch) & 255)
+    return invalid("csc_storage and scratch must be 256-byte aligned");
+  size_t need_csc, need_scratch;
+  transpose_sizes(g->n, g->nnz, g->edge_w != nullptr, &need_csc, &need_scratch);
+  if (csc_bytes < need_csc || scratch_bytes < need_scratch) {
+    set_error("workspace smaller than dg_graph_transpose_workspace reports");
+    return DG_ERR_WORKSPACE;
+  }
+  if (overlaps(csc_storage, scratch, need_csc < need_scratch ? need_csc : need_scratch))
+    return invalid("csc_storage and scratch overlap");
+  g->transposed = false;
+  if (dg_status_t st = transpose_run(g, csc_storage, scratch, (cudaStream_t)stream)) return st;
+  g->transposed = true;
+  return refresh_heavy(g, false, true, (cudaStream_t)stream);
+}
+
+dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t** rowidx_T,
+                             const float** w_T, const int32_t** perm) {
+  if (!g) return invalid("graph handle is NULL");
+  if (!g->transposed) {
+    set_error("dg_graph_transpose has not been called");
+    return DG_ERR_NOT_TRANSPOSED;
+  }
+  if (colptr) *colptr = g->colptr;
+  if (rowidx_T) *rowidx_T = g->rowidx_T;
+  if (w_T) *w_T = g->w_T;
+  if (perm) *perm = g->perm;
+  return DG_OK;
+}
+
+dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op, float* out,
+                             void* stream) {
+  if (dg_status_t st = check_features(g, H, out, F, op)) return st;
+  ApArgs a{};
+  a.ptr = g->rowptr;
+  a.idx = g->colidx;
+  a.w = g->edge_w;
+  a.node_scale = nullptr;
+  a.X = H;
+  a.Y = out;
+  a.heavy_list = g->heavy_rows;
+  a.heavy_count = g->counters + 0;
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.n = g->n;
+  a.F = F;
+  a.mean_rows = op == DG_OP_MEAN;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
+  a.rows_per_block = (int32_t)g->rows_per_block;
+  return aggregate_run(g, a, (cudaStream_t)stream);
+}
+
+dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t op, float* dH,
+                             void* stream) {
+  if (dg_status_t st = check_features(g, dOut, dH, F, op)) return st;
+  if (!g->transposed) {
+    set_error("dg_aggregate_bwd needs dg_graph_transpose first");
+    return DG_ERR_NOT_TRANSPOSED;
+  }
+  ApArgs a{};
+  a.ptr = g->colptr;
+  a.idx = g->rowidx_T;
+  a.w = g->w_T;
+  a.node_scale = op == DG_OP_MEAN ? g->inv_deg : nullptr;
+  a.X = dOut;
+  a.Y = dH;
+  a.heavy_list = g->heavy_cols;
+  a.heavy_count = g->counters + 1;
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.n = g->n;
+  a.F = F;
+  a.mean_rows = 0;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
+  a.rows_per_block = (int32_t)g->rows_per_block;
+  return aggregate_run(g, a, (cudaStream_t)stream);
+}
+
+size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F) {
+  if (!g || F < 1) return 0;
+  const size_t mat = (((size_t)g->n * (size_t)F * sizeof(float)) + 255) & ~(size_t)255;
+  return 2 * (mat > 0 ? mat : 256);
+}
+
+dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dOut_host,
+                              int32_t F, dg_op_t op, float* out_host, float* dH_host,
+                              void* device_ws, size_t device_ws_bytes, void* stream) {
+  if (!g) return invalid("graph handle is NULL");
+  if (F < 1) return invalid("F must be >= 1");
+  if (!H_host || !out_host) return invalid("H_host or out_host is NULL");
+  if ((dOut_host == nullptr) != (dH_host == nullptr))
+    return invalid("dOut_host and dH_host must both be given or both be NULL");
+  if (!device_ws || ((uintptr_t)device_ws & 255)) return invalid("device_ws is NULL or misaligned");
+  if (device_ws_bytes < dg_aggregate_host_workspace(g, F)) {
+    set_error("device_ws smaller than dg_aggregate_host_workspace reports");
+    return DG_ERR_WORKSPACE;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  const size_t bytes = (size_t)g->n * (size_t)F * sizeof(float);
+  const size_t mat = dg_aggregate_host_workspace(g, F) / 2;
+  float* d_in = reinterpret_cast<float*>(device_ws);
+  float* d_out = reinterpret_cast<float*>(static_cast<char*>(device_ws) + mat);
+  if (bytes) DG_CUDA(cudaMemcpyAsync(d_in, H_host, bytes, cudaMemcpyHostToDevice, s));
+  if (dg_status_t st = dg_aggregate_fwd(g, d_in, F, op, d_out, stream)) return st;
+  if (bytes) DG_CUDA(cudaMemcpyAsync(out_host, d_out, bytes, cudaMemcpyDeviceToHost, s));
+  if (dOut_host) {
+    if (bytes) DG_CUDA(cudaMemcpyAsync(d_in, dOut_host, bytes, cudaMemcpyHostToDevice, s));
+    if (dg_status_t st = dg_aggregate_bwd(g, d_in, F, op, d_out, stream)) return st;
+    if (bytes) DG_CUDA(cudaMemcpyAsync(dH_host, d_out, bytes, cudaMemcpyDeviceToHost, s));
+  }
+  return DG_OK;
+}
+
+dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
+  if (!g || !name) return invalid("graph handle or name is NULL");
+  if (!strcmp(name, "heavy_threshold")) {
+    if (value < 64 || value > (1 << 30)) return invalid("heavy_threshold must be in [64, 2^30]");
+    g->heavy_threshold = value;
+    if (dg_status_t st = refresh_heavy(g, true, true, 0)) return st;
+    DG_CUDA(cudaStreamSynchronize(0));
+    return DG_OK;
+  }
+  if (!strcmp(name, "slice_features")) {
+    if (value < 0 || value > (1 << 20)) return invalid("slice_features must be in [0, 2^20]");
+    g->slice_features = value;
+    return DG_OK;
+  }
+  if (!strcmp(name, "rows_per_block")) {
+    if (value < 1 || value > 4096) return invalid("rows_per_block must be in [1, 4096]");
+    g->rows_per_block = value;
+    return DG_OK;
+  }
+  return invalid("unknown parameter name");
+}
+
+dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
+  if (!g || !name || !value) return invalid("graph handle, name or value is NULL");
+  if (!strcmp(name, "heavy_threshold")) { *value = g->heavy_threshold; return DG_OK; }
+  if (!strcmp(name, "slice_features")) { *value = g->slice_features; return DG_OK; }
+  if (!strcmp(name, "rows_per_block")) { *value = g->rows_per_block; return DG_OK; }
+  return invalid("unknown parameter name");
+}
+
+int64_t dg_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* dg_last_error(void) { return g_last_error.c_str(); }
+
+const char* dg_version(void) { return "libdgagg 0.1 sm_100a"; }
+
+}  // extern "C"

@@ -1,0 +1,99 @@
+// Graph ingest kernels: 1/in-degree per vertex, the lists of heavy segments, CSR validation.
+// All integer work except the reciprocal; nothing here waits on another block.
+#include "dg_internal.cuh"
+
+namespace dg {
+namespace {
+
+constexpr int kBlock = 256;
+
+__global__ void inv_deg_kernel(const int64_t* __restrict__ rowptr, int64_t n,
+                               float* __restrict__ inv_deg) {
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= n) return;
+  const int64_t d = rowptr[v + 1] - rowptr[v];
+  inv_deg[v] = d > 0 ? 1.0f / (float)d : 0.0f;
+}
+
+// Appends every segment longer than `threshold` to `list`.  The order of the list does not
+// influence any result: each heavy segment is summed by one block on its own.
+__global__ void heavy_list_kernel(const int64_t* __restrict__ ptr, int64_t n, int64_t threshold,
+                                  int32_t* __restrict__ list, int64_t cap,
+                                  int32_t* __restrict__ count) {
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= n) return;
+  if (ptr[v + 1] - ptr[v] > threshold) {
+    const int32_t slot = atomicAdd(count, 1);
+    if (slot < cap) list[slot] = (int32_t)v;
+  }
+}
+
+// flags: bit 0 rowptr[0] != 0, bit 1 rowptr decreasing, bit 2 rowptr[n] != nnz,
+//        bit 3 colidx out of range
+__global__ void validate_rowptr_kernel(const int64_t* __restrict__ rowptr, int64_t n,
+                                       int64_t nnz, int32_t* __restrict__ flags) {
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v > n) return;
+  int f = 0;
+  if (v == 0 && rowptr[0] != 0) f |= 1;
+  if (v < n && rowptr[v + 1] < rowptr[v]) f |= 2;
+  if (v == n && rowptr[n] != nnz) f |= 4;
+  if (f) atomicOr(flags, f);
+}
+
+__global__ void validate_colidx_kernel(const int32_t* __restrict__ colidx, int64_t nnz,
+                                       int64_t n, int32_t* __restrict__ flags) {
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int bad = 0;
+  for (int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; k < nnz; k += stride) {
+    const int32_t u = colidx[k];
+    if (u < 0 || u >= n) bad = 1;
+  }
+  if (bad) atomicOr(flags, 8);
+}
+
+inline unsigned blocks_for(int64_t items) { return (unsigned)((items + kBlock - 1) / kBlock); }
+
+}  // namespace
+
+dg_status_t build_degree_info(Graph* g, cudaStream_t s) {
+  if (g->n == 0) return DG_OK;
+  inv_deg_kernel<<<blocks_for(g->n), kBlock, 0, s>>>(g->rowptr, g->n, g->inv_deg);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
+}
+
+dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, int32_t* list,
+                             int64_t cap, int32_t* count, cudaStream_t s) {
+  DG_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t), s));
+  if (n == 0) return DG_OK;
+  heavy_list_kernel<<<blocks_for(n), kBlock, 0, s>>>(ptr, n, threshold, list, cap, count);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
+}
+
+dg_status_t validate_csr(Graph* g, cudaStream_t s, int* flags_host) {
+  int32_t* flags = g->counters + 2;
+  DG_CUDA(cudaMemsetAsync(flags, 0, sizeof(int32_t), s));
+  validate_rowptr_kernel<<<blocks_for(g->n + 1), kBlock, 0, s>>>(g->rowptr, g->n, g->nnz, flags);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  // rowptr must be sane before colidx is walked up to nnz: stop here if it is not
+  int32_t h = 0;
+  DG_CUDA(cudaMemcpyAsync(&h, flags, sizeof(h), cudaMemcpyDeviceToHost, s));
+  DG_CUDA(cudaStreamSynchronize(s));
+  if (h == 0 && g->nnz > 0) {
+    const unsigned grid = (unsigned)(g->sm_count * 8);
+    validate_colidx_kernel<<<grid, kBlock, 0, s>>>(g->colidx, g->nnz, g->n, flags);
+    DG_CUDA(cudaGetLastError());
+    count_launches(1);
+    DG_CUDA(cudaMemcpyAsync(&h, flags, sizeof(h), cudaMemcpyDeviceToHost, s));
+    DG_CUDA(cudaStreamSynchronize(s));
+  }
+  *flags_host = h;
+  return DG_OK;
+}
+
+}  // namespace dg

@@ -1,0 +1,339 @@
+// CSR -> CSC on the GPU as a stable least-significant-digit radix sort of (key = colidx[k],
+// value = k).  The paper keeps the graph in CSR only (Section 3.1) and leaves the reverse graph
+// of the backward pass implicit; the result here is defined as the stable counting sort of the
+// edge positions by source vertex, which has exactly one correct answer.
+//
+// One pass over a digit of kRadixBits bits is three kernels and never makes one block wait for
+// another:
+//   1. digit_histogram : per tile of kTile keys, the number of keys per digit -> hist[digit][tile]
+//   2. exclusive scan of hist (digit-major, so the scan yields global output offsets):
+//      scan_reduce -> scan_spine (one block) -> scan_apply
+//   3. digit_scatter   : ranks every key inside its tile in input order (match.any inside a warp,
+//      per-warp counters across rounds, a fixed pass across the warps), stages the tile sorted by
+//      digit in shared memory and writes each digit run to its global offset.
+// Stability of every step makes the final order (key, k) ascending.  After the last pass the
+// sorted keys give colptr by boundary detection, and perm gives rowidx_T and w_T by gathers.
+#include "dg_internal.cuh"
+
+namespace dg {
+namespace {
+
+constexpr int kRadixBits = 8;
+constexpr int kRadix = 1 << kRadixBits;
+constexpr int kSortBlock = 256;
+constexpr int kSortWarps = kSortBlock / 32;
+constexpr int kItems = 16;                       // keys per thread
+constexpr int kTile = kSortBlock * kItems;       // 4096 keys per block
+constexpr int kScanBlock = 256;
+constexpr int kScanItems = 16;
+constexpr int kScanChunk = kScanBlock * kScanItems;
+constexpr unsigned kFull = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t digit_of(uint32_t key, int shift) {
+  return (key >> shift) & (kRadix - 1);
+}
+
+__global__ void __launch_bounds__(kSortBlock)
+digit_histogram(const uint32_t* __restrict__ keys, int64_t count, int shift, int64_t tiles,
+                uint32_t* __restrict__ hist) {
+  __shared__ uint32_t h[kRadix];
+  h[threadIdx.x] = 0;
+  __syncthreads();
+  const int64_t base = (int64_t)blockIdx.x * kTile;
+#pragma unroll 4
+  for (int i = 0; i < kItems; ++i) {
+    const int64_t k = base + i * kSortBlock + threadIdx.x;
+    if (k < count) atomicAdd(&h[digit_of(keys[k], shift)], 1u);
+  }
+  __syncthreads();
+  hist[(int64_t)threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];
+}
+
+// ---- exclusive scan of a uint32 array of length m (in place), three kernels ----
+__device__ __forceinline__ uint32_t block_exclusive_scan(uint32_t v, uint32_t* total) {
+  __shared__ uint32_t warp_sums[kScanBlock / 32];
+  __shared__ uint32_t block_total;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const uint32_t t = __shfl_up_sync(kFull, inc, d);
+    if (lane >= d) inc += t;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    uint32_t w = lane < kScanBlock / 32 ? warp_sums[lane] : 0;
+    uint32_t winc = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const uint32_t t = __shfl_up_sync(kFull, winc, d);
+      if (lane >= d) winc += t;
+    }
+    if (lane < kScanBlock / 32) warp_sums[lane] = winc - w;
+    if (lane == kScanBlock / 32 - 1) block_total = winc;
+  }
+  __syncthreads();
+  const uint32_t r = inc - v + warp_sums[warp];
+  *total = block_total;
+  __syncthreads();  // the shared arrays may be reused by the next call
+  return r;
+}
+
+__global__ void __launch_bounds__(kScanBlock)
+scan_reduce(const uint32_t* __restrict__ data, int64_t m, uint32_t* __restrict__ chunk_sums) {
+  const int64_t base = (int64_t)blockIdx.x * kScanChunk + (int64_t)threadIdx.x * kScanItems;
+  uint32_t s = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i)
+    if (base + i < m) s += data[base + i];
+  uint32_t total;
+  block_exclusive_scan(s, &total);
+  if (threadIdx.x == 0) chunk_sums[blockIdx.x] = total;
+}
+
+__global__ void __launch_bounds__(kScanBlock)
+scan_spine(uint32_t* __restrict__ chunk_sums, int64_t chunks) {
+  uint32_t carry = 0;
+  for (int64_t base = 0; base < chunks; base += kScanBlock) {
+    const int64_t i = base + threadIdx.x;
+    const uint32_t v = i < chunks ? chunk_sums[i] : 0;
+    uint32_t total;
+    const uint32_t ex = block_exclusive_scan(v, &total);
+    if (i < chunks) chunk_sums[i] = carry + ex;
+    carry += total;
+  }
+}
+
+__global__ void __launch_bounds__(kScanBlock)
+scan_apply(uint32_t* __restrict__ data, int64_t m, const uint32_t* __restrict__ chunk_sums) {
+  const int64_t base = (int64_t)blockIdx.x * kScanChunk + (int64_t)threadIdx.x * kScanItems;
+  uint32_t v[kScanItems];
+  uint32_t s = 0;
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    v[i] = base + i < m ? data[base + i] : 0;
+    s += v[i];
+  }
+  uint32_t total;
+  uint32_t run = block_exclusive_scan(s, &total) + chunk_sums[blockIdx.x];
+#pragma unroll
+  for (int i = 0; i < kScanItems; ++i) {
+    if (base + i < m) data[base + i] = run;
+    run += v[i];
+  }
+}
+
+// ---- stable scatter of one tile ----
+// vals_in == nullptr means "the value of key k is k" (first pass).  keys_out may be nullptr when
+// the sorted keys are not needed (never the case for the last pass, which feeds colptr).
+__global__ void __launch_bounds__(kSortBlock)
+digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
+              int64_t count, int shift, int64_t tiles, const uint32_t* __restrict__ offsets,
+              uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out) {
+  __shared__ uint32_t warp_cnt[kSortWarps][kRadix];
+  __shared__ uint32_t digit_base[kRadix];
+  __shared__ uint32_t global_base[kRadix];
+  __shared__ uint32_t skeys[kTile];
+  __shared__ uint32_t svals[kTile];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned lt_mask = (1u << lane) - 1u;
+  const int64_t tile_base = (int64_t)blockIdx.x * kTile;
+  const int64_t remaining = count - tile_base;
+  const int tile_count = remaining < kTile ? (int)remaining : kTile;
+
+  for (int w = 0; w < kSortWarps; ++w) warp_cnt[w][threadIdx.x] = 0;
+  __syncthreads();
+
+  // Warp `warp` owns keys [warp*512, warp*512+512) of the tile, 32 consecutive keys per round,
+  // so (warp, round, lane) order is input order.
+  uint32_t key[kItems];
+  uint32_t val[kItems];
+  uint16_t rank[kItems];
+#pragma unroll
+  for (int r = 0; r < kItems; ++r) {
+    const int local = warp * (32 * kItems) + r * 32 + lane;
+    const bool valid = local < tile_count;
+    key[r] = valid ? keys_in[tile_base + local] : 0u;
+    val[r] = valid ? (vals_in ? vals_in[tile_base + local] : (uint32_t)(tile_base + local)) : 0u;
+    const uint32_t d = valid ? digit_of(key[r], shift) : (uint32_t)kRadix;  // kRadix = "none"
+    const unsigned peers = __match_any_sync(kFull, d);
+    const int leader = __ffs(peers) - 1;
+    uint32_t before = 0;
+    if (valid && lane == leader) {
+      before = warp_cnt[warp][d];
+      warp_cnt[warp][d] = before + __popc(peers);
+    }
+    before = __shfl_sync(kFull, before, leader);
+    rank[r] = (uint16_t)(before + __popc(peers & lt_mask));
+    __syncwarp();
+  }
+  __syncthreads();
+
+  // thread t owns digit t: exclusive prefix over the warps, then over the digits
+  {
+    const int d = threadIdx.x;
+    uint32_t run = 0;
+#pragma unroll
+    for (int w = 0; w < kSortWarps; ++w) {
+      const uint32_t c = warp_cnt[w][d];
+      warp_cnt[w][d] = run;
+      run += c;
+    }
+    uint32_t total;
+    digit_base[d] = block_exclusive_scan(run, &total);
+    global_base[d] = offsets[(int64_t)d * tiles + blockIdx.x];
+  }
+  __syncthreads();
+
+#pragma unroll
+  for (int r = 0; r < kItems; ++r) {
+    const int local = warp * (32 * kItems) + r * 32 + lane;
+    if (local < tile_count) {
+      const uint32_t d = digit_of(key[r], shift);
+      const uint32_t pos = digit_base[d] + warp_cnt[warp][d] + rank[r];
+      skeys[pos] = key[r];
+      svals[pos] = val[r];
+    }
+  }
+  __syncthreads();
+
+  for (int i = threadIdx.x; i < tile_count; i += kSortBlock) {
+    const uint32_t k = skeys[i];
+    const uint32_t d = digit_of(k, shift);
+    const uint32_t dst = global_base[d] + ((uint32_t)i - digit_base[d]);
+    if (keys_out) keys_out[dst] = k;
+    vals_out[dst] = svals[i];
+  }
+}
+
+// colptr[u] = first position q whose sorted key is >= u.  Thread q fills the ids between the
+// key before it and its own key; thread nnz closes the array up to n.
+__global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int64_t nnz,
+                                        int64_t n, int64_t* __restrict__ colptr) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q > nnz) return;
+  const int64_t prev = q > 0 ? (int64_t)sorted[q - 1] : -1;
+  int64_t cur = q < nnz ? (int64_t)sorted[q] : n;
+  if (cur > n) cur = n;  // an id outside [0, n) must not turn into a write outside colptr
+  for (int64_t u = prev + 1; u <= cur; ++u) colptr[u] = q;
+}
+
+// rowidx_T[q] = the row r with rowptr[r] <= perm[q] < rowptr[r+1];  w_T[q] = edge_w[perm[q]].
+__global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64_t nnz,
+                                        const int64_t* __restrict__ rowptr, int64_t n,
+                                        const float* __restrict__ edge_w,
+                                        int32_t* __restrict__ rowidx_T, float* __restrict__ w_T) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= nnz) return;
+  const int64_t k = perm[q];
+  int64_t lo = 0, hi = n;  // invariant: rowptr[lo] <= k < rowptr[hi]
+  while (hi - lo > 1) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (__ldg(rowptr + mid) <= k) lo = mid; else hi = mid;
+  }
+  rowidx_T[q] = (int32_t)lo;
+  if (edge_w) w_T[q] = edge_w[k];
+}
+
+inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct Layout {
+  // csc storage
+  size_t colptr_off, rowidx_off, perm_off, w_off, csc_bytes;
+  // scratch
+  size_t keys_a_off, keys_b_off, vals_off, hist_off, sums_off, scratch_bytes;
+  int64_t tiles, hist_len, chunks;
+  int passes;
+};
+
+Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
+  Layout L{};
+  size_t o = 0;
+  L.colptr_off = o; o += align256((size_t)(n + 1) * 8);
+  L.rowidx_off = o; o += align256((size_t)nnz * 4);
+  L.perm_off = o;   o += align256((size_t)nnz * 4);
+  L.w_off = o;      o += weighted ? align256((size_t)nnz * 4) : 0;
+  L.csc_bytes = o > 0 ? o : 256;
+  int bits = 1;
+  while (bits < 31 && ((int64_t)1 << bits) < n) ++bits;
+  L.passes = (bits + kRadixBits - 1) / kRadixBits;
+  L.tiles = (nnz + kTile - 1) / kTile;
+  L.hist_len = L.tiles * kRadix;
+  L.chunks = (L.hist_len + kScanChunk - 1) / kScanChunk;
+  o = 0;
+  L.keys_a_off = o; o += align256((size_t)nnz * 4);
+  L.keys_b_off = o; o += align256((size_t)nnz * 4);
+  L.vals_off = o;   o += align256((size_t)nnz * 4);
+  L.hist_off = o;   o += align256((size_t)L.hist_len * 4);
+  L.sums_off = o;   o += align256((size_t)(L.chunks > 0 ? L.chunks : 1) * 4);
+  L.scratch_bytes = o > 0 ? o : 256;
+  return L;
+}
+
+}  // namespace
+
+void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
+                     size_t* scratch_bytes) {
+  const Layout L = make_layout(n, nnz, weighted);
+  *csc_bytes = L.csc_bytes;
+  *scratch_bytes = L.scratch_bytes;
+}
+
+dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
+  const int64_t n = g->n, nnz = g->nnz;
+  const bool weighted = g->edge_w != nullptr;
+  const Layout L = make_layout(n, nnz, weighted);
+  char* cb = static_cast<char*>(csc);
+  char* sb = static_cast<char*>(scratch);
+  int64_t* colptr = reinterpret_cast<int64_t*>(cb + L.colptr_off);
+  int32_t* rowidx_T = reinterpret_cast<int32_t*>(cb + L.rowidx_off);
+  uint32_t* perm = reinterpret_cast<uint32_t*>(cb + L.perm_off);
+  float* w_T = weighted ? reinterpret_cast<float*>(cb + L.w_off) : nullptr;
+  uint32_t* keys_buf[2] = {reinterpret_cast<uint32_t*>(sb + L.keys_a_off),
+                           reinterpret_cast<uint32_t*>(sb + L.keys_b_off)};
+  uint32_t* vals_tmp = reinterpret_cast<uint32_t*>(sb + L.vals_off);
+  uint32_t* hist = reinterpret_cast<uint32_t*>(sb + L.hist_off);
+  uint32_t* sums = reinterpret_cast<uint32_t*>(sb + L.sums_off);
+
+  if (nnz == 0) {
+    DG_CUDA(cudaMemsetAsync(colptr, 0, (size_t)(n + 1) * 8, s));
+  } else {
+    const uint32_t* keys_in = reinterpret_cast<const uint32_t*>(g->colidx);
+    const uint32_t* vals_in = nullptr;
+    for (int p = 0; p < L.passes; ++p) {
+      const int shift = p * kRadixBits;
+      // value buffers alternate so that the last pass lands in perm
+      uint32_t* vals_out = ((L.passes - 1 - p) % 2 == 0) ? perm : vals_tmp;
+      uint32_t* keys_out = keys_buf[p % 2];
+      digit_histogram<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, nnz, shift, L.tiles, hist);
+      DG_CUDA(cudaGetLastError());
+      scan_reduce<<<(unsigned)L.chunks, kScanBlock, 0, s>>>(hist, L.hist_len, sums);
+      DG_CUDA(cudaGetLastError());
+      scan_spine<<<1, kScanBlock, 0, s>>>(sums, L.chunks);
+      DG_CUDA(cudaGetLastError());
+      scan_apply<<<(unsigned)L.chunks, kScanBlock, 0, s>>>(hist, L.hist_len, sums);
+      DG_CUDA(cudaGetLastError());
+      digit_scatter<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, vals_in, nnz, shift,
+                                                            L.tiles, hist, keys_out, vals_out);
+      DG_CUDA(cudaGetLastError());
+      count_launches(5);
+      keys_in = keys_out;
+      vals_in = vals_out;
+    }
+    const unsigned b1 = (unsigned)((nnz + 1 + 255) / 256);
+    colptr_from_sorted_keys<<<b1, 256, 0, s>>>(keys_in, nnz, n, colptr);
+    DG_CUDA(cudaGetLastError());
+    const unsigned b2 = (unsigned)((nnz + 255) / 256);
+    gather_rows_and_weights<<<b2, 256, 0, s>>>(perm, nnz, g->rowptr, n, g->edge_w, rowidx_T, w_T);
+    DG_CUDA(cudaGetLastError());
+    count_launches(2);
+  }
+  g->colptr = colptr;
+  g->rowidx_T = rowidx_T;
+  g->perm = reinterpret_cast<const int32_t*>(perm);
+  g->w_T = w_T;
+  return DG_OK;
+}
+
+}  // namespace dg

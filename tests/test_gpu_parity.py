@@ -1,0 +1,253 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element.
+
+fp32 outputs must satisfy |gpu - ref| <= 1e-5 * sum|terms| + 1e-7 per element; the CSC arrays
+(colptr, rowidx_T, perm) and the copied weights must be bit-exact.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_06700_b200 import binding, synth
+from parity_util import (assert_within_bound, check_fwd_bwd, check_transpose, make_graph, to_np)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def host_csr(sg):
+    return (to_np(sg.rowptr), to_np(sg.colidx), to_np(sg.edge_w))
+
+
+def csr_graph(n, rows, device=DEV, weights=None):
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    col = []
+    for v in range(n):
+        col.extend(rows[v])
+        rowptr[v + 1] = len(col)
+    colidx = np.asarray(col, dtype=np.int32)
+    w = None if weights is None else torch.as_tensor(weights, dtype=torch.float32, device=device)
+    g = binding.dg_graph_create(n, len(col), torch.as_tensor(rowptr, device=device),
+                                torch.as_tensor(colidx, device=device), w)
+    return g, rowptr, colidx
+
+
+# ------------------------------------------------------------------ tiny: every combination
+@pytest.fixture(scope="module")
+def tiny():
+    return synth.make("tiny")
+
+
+@pytest.mark.parametrize("weighted", [True, False])
+def test_tiny_transpose_bit_exact(tiny, weighted):
+    sg = tiny if weighted else synth.make("tiny", weighted=False)
+    g = make_graph(sg)
+    g.dg_graph_validate()
+    check_transpose(g, *host_csr(sg))
+
+
+@pytest.mark.parametrize("F", [64, 8, 100, 602, 256, 128, 1, 3, 6, 130, 1028])
+@pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
+@pytest.mark.parametrize("weighted", [True, False])
+def test_tiny_forward_backward(tiny, F, op, weighted):
+    sg = tiny if weighted else synth.make("tiny", weighted=False)
+    g = make_graph(sg)
+    csc = check_transpose(g, *host_csr(sg))
+    H = synth.features(sg.n, F, 100 + F, DEV)
+    G = synth.features(sg.n, F, 200 + F, DEV)
+    check_fwd_bwd(g, host_csr(sg), H, G, op, csc)
+
+
+def test_tiny_deterministic_bits(tiny):
+    g = make_graph(tiny)
+    g.dg_graph_transpose()
+    H = synth.features(tiny.n, 64, 1, DEV)
+    a = g.dg_aggregate_fwd(H, binding.DG_OP_MEAN).clone()
+    b = g.dg_aggregate_fwd(H, binding.DG_OP_MEAN)
+    c = g.dg_aggregate_bwd(H, binding.DG_OP_MEAN).clone()
+    d = g.dg_aggregate_bwd(H, binding.DG_OP_MEAN)
+    assert torch.equal(a, b) and torch.equal(c, d)
+
+
+@pytest.mark.parametrize("slice_f,heavy,rows_per_block", [(16, 64, 1), (32, 64, 8), (0, 128, 64),
+                                                         (600, 1024, 32), (4, 4096, 3)])
+def test_tiny_launch_shapes(tiny, slice_f, heavy, rows_per_block):
+    """Feature slicing, the heavy-segment path and the block shape change the launch, not the
+    result (columns of the tiny graph reach 488 entries, above the lowered heavy threshold)."""
+    g = make_graph(tiny)
+    g.dg_graph_set_param("heavy_threshold", heavy)
+    g.dg_graph_set_param("slice_features", slice_f)
+    g.dg_graph_set_param("rows_per_block", rows_per_block)
+    assert g.dg_graph_get_param("heavy_threshold") == heavy
+    csc = check_transpose(g, *host_csr(tiny))
+    for F in (64, 602, 10):
+        H = synth.features(tiny.n, F, 5, DEV)
+        G = synth.features(tiny.n, F, 6, DEV)
+        check_fwd_bwd(g, host_csr(tiny), H, G, binding.DG_OP_MEAN, csc)
+
+
+def test_unaligned_feature_pointers(tiny):
+    """Matrices that start 4 or 8 bytes off a 16-byte boundary take the narrower vector paths."""
+    g = make_graph(tiny)
+    csc = check_transpose(g, *host_csr(tiny))
+    for F, shift in ((64, 1), (64, 2), (602, 1)):
+        base = synth.features(tiny.n * F + 4, 1, 9, DEV).flatten()
+        H = base[shift:shift + tiny.n * F].view(tiny.n, F)
+        G = synth.features(tiny.n, F, 10, DEV)
+        outbuf = torch.empty(tiny.n * F + 4, device=DEV)
+        out = outbuf[shift:shift + tiny.n * F].view(tiny.n, F)
+        g.dg_aggregate_fwd(H, binding.DG_OP_SUM, out=out)
+        torch.cuda.synchronize()
+        ref, mag = oracle.ap_forward(*host_csr(tiny), to_np(H.contiguous()), oracle.OP_SUM)
+        assert_within_bound(to_np(out), ref, mag, f"unaligned F={F} shift={shift}")
+        check_fwd_bwd(g, host_csr(tiny), H.contiguous(), G, binding.DG_OP_SUM, csc)
+
+
+# ------------------------------------------------------------------ closed forms, degenerate
+def test_identity_and_ring_bit_exact():
+    n, F = 1000, 96
+    H = synth.features(n, F, 3, DEV)
+    g, *_ = csr_graph(n, [[v] for v in range(n)])
+    g.dg_graph_transpose()
+    for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+        assert torch.equal(g.dg_aggregate_fwd(H, op), H)
+        assert torch.equal(g.dg_aggregate_bwd(H, op), H)
+    g, *_ = csr_graph(n, [[(v - 1) % n] for v in range(n)])
+    g.dg_graph_transpose()
+    assert torch.equal(g.dg_aggregate_fwd(H, binding.DG_OP_SUM), torch.roll(H, 1, 0))
+    assert torch.equal(g.dg_aggregate_bwd(H, binding.DG_OP_SUM), torch.roll(H, -1, 0))
+
+
+@pytest.mark.parametrize("F", [8, 100, 602])
+def test_star_graph_heavy_row_and_column(F):
+    """Vertex 0 pulls from every other vertex (one CSR row of n-1 entries, a heavy row), and
+    every other vertex pulls from vertex 1 (one CSC column of n-1 entries)."""
+    n = 6000
+    rows = [list(range(1, n))] + [[1] for _ in range(n - 1)]
+    w = np.random.default_rng(0).random(2 * (n - 1)).astype(np.float32)
+    g, rowptr, colidx = csr_graph(n, rows, weights=w)
+    csc = check_transpose(g, rowptr, colidx, w)
+    H = synth.features(n, F, 11, DEV)
+    G = synth.features(n, F, 12, DEV)
+    for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+        check_fwd_bwd(g, (rowptr, colidx, w), H, G, op, csc)
+
+
+def test_empty_rows_give_zeros_and_empty_graphs_work():
+    n, F = 300, 20
+    rows = [[] for _ in range(n)]
+    rows[7] = [1, 2, 3]
+    g, rowptr, colidx = csr_graph(n, rows)
+    g.dg_graph_transpose()
+    H = synth.features(n, F, 13, DEV)
+    out = torch.full((n, F), float("nan"), device=DEV)   # the library overwrites, never reads out
+    g.dg_aggregate_fwd(H, binding.DG_OP_MEAN, out=out)
+    assert torch.all(out[:7] == 0) and torch.all(out[8:] == 0)
+    assert torch.allclose(out[7], H[1:4].mean(0), atol=1e-6)
+    # nnz = 0
+    g0 = binding.dg_graph_create(5, 0, torch.zeros(6, dtype=torch.int64, device=DEV),
+                                 torch.zeros(0, dtype=torch.int32, device=DEV), None)
+    g0.dg_graph_validate()
+    g0.dg_graph_transpose()
+    colptr, rowidx_T, w_T, perm = g0.dg_graph_get_csc()
+    assert torch.all(colptr == 0) and rowidx_T.numel() == 0 and w_T is None
+    H5 = synth.features(5, 4, 1, DEV)
+    assert torch.all(g0.dg_aggregate_fwd(H5, binding.DG_OP_SUM) == 0)
+    assert torch.all(g0.dg_aggregate_bwd(H5, binding.DG_OP_MEAN) == 0)
+    # n = 0
+    g00 = binding.dg_graph_create(0, 0, torch.zeros(1, dtype=torch.int64, device=DEV),
+                                  torch.zeros(0, dtype=torch.int32, device=DEV), None)
+    g00.dg_graph_transpose()
+    e = torch.zeros((0, 4), device=DEV)
+    assert g00.dg_aggregate_fwd(e, binding.DG_OP_SUM).shape == (0, 4)
+
+
+def test_unsorted_rows_duplicates_and_self_loops():
+    rng = np.random.default_rng(21)
+    n, nnz, F = 500, 20000, 36
+    dst = np.sort(rng.integers(0, n, nnz))
+    src = rng.integers(0, n, nnz).astype(np.int32)        # unsorted inside rows, with repeats
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.add.at(rowptr, dst + 1, 1)
+    rowptr = np.cumsum(rowptr)
+    w = rng.random(nnz).astype(np.float32)
+    g = binding.dg_graph_create(n, nnz, torch.as_tensor(rowptr, device=DEV),
+                                torch.as_tensor(src, device=DEV), torch.as_tensor(w, device=DEV))
+    csc = check_transpose(g, rowptr, src, w)
+    H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
+    check_fwd_bwd(g, (rowptr, src, w), H, G, binding.DG_OP_MEAN, csc)
+
+
+# ------------------------------------------------------------------ errors never trap
+def test_error_statuses(tiny):
+    g = make_graph(tiny)
+    H = synth.features(tiny.n, 64, 1, DEV)
+    with pytest.raises(binding.DgError) as e:
+        g.dg_aggregate_bwd(H, binding.DG_OP_SUM)
+    assert e.value.status == binding.DG_ERR_NOT_TRANSPOSED
+    with pytest.raises(binding.DgError) as e:
+        g.dg_graph_get_csc()
+    assert e.value.status == binding.DG_ERR_NOT_TRANSPOSED
+    with pytest.raises(binding.DgError) as e:
+        g.dg_aggregate_fwd(H, binding.DG_OP_SUM, out=H)           # aliasing
+    assert e.value.status == binding.DG_ERR_INVALID_ARG
+    with pytest.raises(binding.DgError) as e:
+        g.dg_aggregate_fwd(H, 7)                                   # bad op
+    assert e.value.status == binding.DG_ERR_INVALID_ARG
+    small = torch.empty(256, dtype=torch.uint8, device=DEV)
+    with pytest.raises(binding.DgError) as e:
+        g.dg_graph_transpose(csc_storage=small)
+    assert e.value.status == binding.DG_ERR_WORKSPACE
+    with pytest.raises(binding.DgError):
+        g.dg_graph_set_param("no_such_knob", 1)
+    # a malformed CSR is reported by validate, not by a fault
+    bad_col = tiny.colidx.clone().to(DEV)
+    bad_col[5] = tiny.n + 3
+    gb = binding.dg_graph_create(tiny.n, tiny.nnz, tiny.rowptr.to(DEV), bad_col, None)
+    with pytest.raises(binding.DgError) as e:
+        gb.dg_graph_validate()
+    assert e.value.status == binding.DG_ERR_INVALID_GRAPH
+    bad_ptr = tiny.rowptr.clone().to(DEV)
+    bad_ptr[10] = bad_ptr[11] + 1
+    gp = binding.dg_graph_create(tiny.n, tiny.nnz, bad_ptr, tiny.colidx.to(DEV), None)
+    with pytest.raises(binding.DgError) as e:
+        gp.dg_graph_validate()
+    assert e.value.status == binding.DG_ERR_INVALID_GRAPH
+    # the context is still healthy
+    g.dg_graph_transpose()
+    g.dg_aggregate_bwd(H, binding.DG_OP_SUM)
+    torch.cuda.synchronize()
+
+
+def test_host_entry_point(tiny):
+    g = make_graph(tiny)
+    g.dg_graph_transpose()
+    F = 64
+    H = synth.features(tiny.n, F, 1).pin_memory()
+    G = synth.features(tiny.n, F, 2).pin_memory()
+    out = torch.empty_like(H).pin_memory()
+    dH = torch.empty_like(H).pin_memory()
+    ws = torch.empty(g.dg_aggregate_host_workspace(F), dtype=torch.uint8, device=DEV)
+    g.dg_aggregate_host(H, G, binding.DG_OP_MEAN, out, dH, ws)
+    torch.cuda.synchronize()
+    assert torch.equal(out, g.dg_aggregate_fwd(H.to(DEV), binding.DG_OP_MEAN).cpu())
+    assert torch.equal(dH, g.dg_aggregate_bwd(G.to(DEV), binding.DG_OP_MEAN).cpu())
+
+
+# ------------------------------------------------------------------ mid-size workloads, in full
+@pytest.mark.parametrize("name,scale,F,ops", [
+    ("reddit_like", 0.02, 602, (binding.DG_OP_MEAN,)),
+    ("products_like", 0.02, 100, (binding.DG_OP_SUM, binding.DG_OP_MEAN)),
+    ("proteins_like", 0.02, 64, (binding.DG_OP_SUM,)),
+    ("papers_like", 0.002, 128, (binding.DG_OP_SUM,)),
+])
+def test_scaled_workloads_full_comparison(name, scale, F, ops):
+    """Several thousand tiles with ragged tails, compared in full with the oracle."""
+    sg = synth.make(name, device=DEV, scale=scale)
+    g = make_graph(sg)
+    g.dg_graph_validate()
+    csc = check_transpose(g, *host_csr(sg))
+    H = synth.features(sg.n, F, 31, DEV)
+    G = synth.features(sg.n, F, 32, DEV)
+    for op in ops:
+        check_fwd_bwd(g, host_csr(sg), H, G, op, csc)
