@@ -16,7 +16,7 @@
  *     ordinary process memory; the library never takes ownership of a caller's buffer;
  *   - `stream` is a CUDA stream handle (cudaStream_t / CUstream passed as void*); NULL is the
  *     legacy default stream.  Calls that take a stream only enqueue work on it;
- *   - feature matrices are dense, row-major, fp32, leading dimension F;
+ *   - feature matrices are dense, row-major, fp32, leading dimension F, 1 <= F <= 2^20;
  *   - rowptr/colptr are int64, vertex ids are int32 (n < 2^31), nnz < 2^31;
  *   - no call aborts, traps or waits without bound on the device.
  */
@@ -141,7 +141,8 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  * Tuning knobs (defaults come from the device's L2 size and SM count):
  *   "heavy_threshold"  rows longer than this are summed by a whole thread block
  *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
- *   "rows_per_block"   destination rows per thread block in the light-row kernel
+ *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
+ *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows)
  * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.
  */
 dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);

@@ -5,10 +5,13 @@
 // source blocking (Algorithm 2) plays on a CPU cache.
 //
 // Work decomposition
-//   light segments (length <= heavy_threshold): one warp per segment.  Lanes are spread along
-//     the feature dimension with 16-, 8- or 4-byte vector loads.  When a row slice needs fewer
-//     than 32 vectors the warp is cut into groups of G lanes and the groups take different
-//     edges of the same segment; their partial sums are combined by a fixed shuffle tree.
+//   light segments (length <= heavy_threshold): every warp owns rows_per_warp consecutive
+//     segments and reads their indices as one contiguous stream of 32-edge batches (one edge
+//     per lane, next batch prefetched), so short rows share coalesced index loads.  Lanes are
+//     spread along the feature dimension with 16-, 8- or 4-byte vector loads.  When a row slice
+//     needs fewer than 32 vectors the warp is cut into groups of G lanes and the groups take
+//     different edges of the same segment; their partial sums are combined by a fixed shuffle
+//     tree.  U load steps per lane are in flight before the first add.
 //   heavy segments: one thread block per segment (the first blocks of the same launch loop over
 //     the heavy list); the 8 warps take interleaved batches of 32 edges and combine in shared
 //     memory in warp order.
@@ -28,11 +31,13 @@ template <> struct Vec<1> { using T = float; };
 template <> struct Vec<2> { using T = float2; };
 template <> struct Vec<4> { using T = float4; };
 
-__device__ __forceinline__ float ldg_vec(const float* p, float) { return __ldg(p); }
-__device__ __forceinline__ float2 ldg_vec(const float* p, float2) {
+__device__ __forceinline__ float ldg_vec(const char* p, float) {
+  return __ldg(reinterpret_cast<const float*>(p));
+}
+__device__ __forceinline__ float2 ldg_vec(const char* p, float2) {
   return __ldg(reinterpret_cast<const float2*>(p));
 }
-__device__ __forceinline__ float4 ldg_vec(const float* p, float4) {
+__device__ __forceinline__ float4 ldg_vec(const char* p, float4) {
   return __ldg(reinterpret_cast<const float4*>(p));
 }
 __device__ __forceinline__ void zero(float& a) { a = 0.f; }
@@ -71,13 +76,15 @@ __device__ __forceinline__ void st_smem(float* p, float4 v) {
   p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
 }
 
-// Loads the neighbour id and the per-edge factor of edge k (k < hi), else a neutral pair.
+// Loads the neighbour id and the per-edge factor of the edge at position b + lane of the
+// index stream (neutral values at or beyond `end`).
 template <bool SCALED>
-__device__ __forceinline__ void load_edge(const ApArgs& a, int64_t k, int64_t hi, int32_t& u,
-                                          float& s) {
+__device__ __forceinline__ void load_batch(const ApArgs& a, int64_t b, int end, int lane,
+                                           int32_t& u, float& s) {
   u = 0;
   s = 0.f;
-  if (k < hi) {
+  const int64_t k = b + lane;
+  if (k < end) {
     u = __ldcs(a.idx + k);
     if (SCALED) {
       s = a.w ? __ldcs(a.w + k) : 1.f;
@@ -86,67 +93,77 @@ __device__ __forceinline__ void load_edge(const ApArgs& a, int64_t k, int64_t hi
   }
 }
 
-// Sums the edges of [lo, hi) that fall into batches first, first+step, ... (32 edges each) into
-// acc.  Within a batch, lane group `grp` takes edges grp, grp+NG, ...; U edges are in flight
-// per group.
+template <int VEC, int G, int CPL>
+struct Shape {
+  static constexpr int NG = 32 / G;  // edges one warp-wide load instruction covers
+  static constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : 2);
+  static constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;  // load steps in flight per lane
+};
+
+// Adds the edges held in lanes [s, e) of the current batch (cur_u / cur_s: one edge per lane)
+// into acc.  Lane group `grp` takes edges s+grp, s+grp+NG, ...  Full steps of U*NG edges run
+// without predicates; the ragged end runs once with predicated loads.  xrow[c] is the address
+// of this lane's c-th vector inside row 0 of X.
 template <int VEC, int G, int CPL, bool SCALED>
-__device__ __forceinline__ void accumulate(const ApArgs& a, int64_t lo, int64_t hi, int first,
-                                           int step, int f0, int fend,
-                                           typename Vec<VEC>::T (&acc)[CPL]) {
+__device__ __forceinline__ void add_edges(const char* const (&xrow)[CPL], uint32_t row_bytes,
+                                          int32_t cur_u, float cur_s, int s, int e, int grp,
+                                          typename Vec<VEC>::T (&acc)[CPL]) {
   using V = typename Vec<VEC>::T;
-  constexpr int NG = 32 / G;
-  constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : 2);
-  constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;
-  const int lane = threadIdx.x & 31;
-  const int grp = lane / G;
-  const int c0 = lane % G;
-
-  int foff[CPL];
-  bool fok[CPL];
+  constexpr int NG = Shape<VEC, G, CPL>::NG;
+  constexpr int U = Shape<VEC, G, CPL>::U;
+  int p = s;
+  for (; p + U * NG <= e; p += U * NG) {
+    V v[U][CPL];
+    float sc[U];
 #pragma unroll
-  for (int c = 0; c < CPL; ++c) {
-    foff[c] = f0 + (c0 + c * G) * VEC;
-    fok[c] = foff[c] < fend;
-  }
-
-  int64_t base = lo + (int64_t)first * 32;
-  int32_t my_u, nx_u;
-  float my_s, nx_s;
-  if (base < hi) load_edge<SCALED>(a, base + lane, hi, nx_u, nx_s);
-  for (; base < hi; base += (int64_t)step * 32) {
-    my_u = nx_u;
-    my_s = nx_s;
-    const int64_t nbase = base + (int64_t)step * 32;
-    if (nbase < hi) load_edge<SCALED>(a, nbase + lane, hi, nx_u, nx_s);
-    const int cnt = (hi - base) < 32 ? (int)(hi - base) : 32;
-    for (int e0 = 0; e0 < cnt; e0 += U * NG) {
-      V v[U][CPL];
-      float s[U];
+    for (int j = 0; j < U; ++j) {
+      const int src = p + j * NG + grp;
+      const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src);
+      if (SCALED) sc[j] = __shfl_sync(kFull, cur_s, src);
+      const uint64_t off = (uint64_t)u * row_bytes;
 #pragma unroll
-      for (int j = 0; j < U; ++j) {
-        const int e = e0 + j * NG + grp;
-        const bool ok = e < cnt;
-        const int32_t u = __shfl_sync(kFull, my_u, e & 31);
-        s[j] = SCALED ? __shfl_sync(kFull, my_s, e & 31) : 1.f;
-        const float* row = a.X + (size_t)u * (size_t)a.F;
+      for (int c = 0; c < CPL; ++c) v[j][c] = ldg_vec(xrow[c] + off, V());
+    }
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          if (ok && fok[c]) v[j][c] = ldg_vec(row + foff[c], V());
-          else zero(v[j][c]);
-        }
-        if (!ok) s[j] = 0.f;
-      }
+    for (int j = 0; j < U; ++j) {
 #pragma unroll
-      for (int j = 0; j < U; ++j) {
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          if (SCALED) fma(acc[c], s[j], v[j][c]);
-          else add(acc[c], v[j][c]);
-        }
+      for (int c = 0; c < CPL; ++c) {
+        if (SCALED) fma(acc[c], sc[j], v[j][c]);
+        else add(acc[c], v[j][c]);
       }
     }
   }
-  // combine the lane groups (fixed tree)
+  if (p < e) {
+    V v[U][CPL];
+    float sc[U];
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+      const int src = p + j * NG + grp;
+      const bool ok = src < e;
+      const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src & 31);
+      sc[j] = SCALED ? __shfl_sync(kFull, cur_s, src & 31) : 1.f;
+      if (!ok) sc[j] = 0.f;
+      const uint64_t off = (uint64_t)u * row_bytes;
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        if (ok) v[j][c] = ldg_vec(xrow[c] + off, V());
+        else zero(v[j][c]);
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < U; ++j) {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        if (SCALED) fma(acc[c], sc[j], v[j][c]);
+        else add(acc[c], v[j][c]);
+      }
+    }
+  }
+}
+
+// Sums the partial results of the lane groups into group 0 (fixed tree).
+template <int VEC, int G, int CPL>
+__device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL]) {
 #pragma unroll
   for (int off = G; off < 32; off <<= 1) {
 #pragma unroll
@@ -155,38 +172,84 @@ __device__ __forceinline__ void accumulate(const ApArgs& a, int64_t lo, int64_t 
 }
 
 // One launch does both roles: blocks [0, heavy_blocks) walk the heavy list (they are scheduled
-// first, so the long segments start early), the remaining blocks take rows_per_block consecutive
-// light segments each.
+// first, so the long segments start early); in the remaining blocks every warp owns
+// rows_per_warp consecutive light segments and streams their indices as one run of 32-edge
+// batches, the next batch always in flight while the current one is summed.
 template <int VEC, int G, int CPL, bool SCALED>
 __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
   using V = typename Vec<VEC>::T;
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
+  const int grp = lane / G;
+  const int c0 = lane % G;
   const int f0 = blockIdx.y * a.slice_f;
   const int fend = min(a.F, f0 + a.slice_f);
-  const int c0 = lane % G;
+  const int width = fend - f0;
+  const int chunks = width / VEC;
+  const uint32_t row_bytes = (uint32_t)a.F * 4u;
+
+  // Lanes whose vector falls beyond the slice re-read vector 0 and never store: the summing
+  // loop then needs no per-lane predicate.
+  const char* xrow[CPL];
+  bool cok[CPL];
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) {
+    const int ci = c0 + c * G;
+    cok[c] = ci < chunks;
+    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * 4u;
+  }
 
   if ((int)blockIdx.x >= heavy_blocks) {
-    const int64_t row0 = (int64_t)(blockIdx.x - heavy_blocks) * a.rows_per_block;
-    const int64_t row1 = min(a.n, row0 + a.rows_per_block);
-    for (int64_t r = row0 + warp; r < row1; r += kWarpsPerBlock) {
-      const int64_t lo = __ldg(a.ptr + r), hi = __ldg(a.ptr + r + 1);
-      const int64_t len = hi - lo;
-      if (len > a.heavy_threshold) continue;  // a heavy block writes this row
+    const int rpw = a.rows_per_warp;
+    const int64_t rb = ((int64_t)(blockIdx.x - heavy_blocks) * kWarpsPerBlock + warp) * rpw;
+    if (rb >= a.n) return;
+    const int nrows = (int)min((int64_t)rpw, a.n - rb);
+    const int my_ptr = lane <= nrows ? (int)__ldg(a.ptr + rb + lane) : 0;
+    const int stream_end = __shfl_sync(kFull, my_ptr, nrows);
+    int b = __shfl_sync(kFull, my_ptr, 0);
+    int32_t cur_u, nxt_u;
+    float cur_s, nxt_s;
+    load_batch<SCALED>(a, b, stream_end, lane, cur_u, cur_s);
+    load_batch<SCALED>(a, (int64_t)b + 32, stream_end, lane, nxt_u, nxt_s);
+    for (int i = 0; i < nrows; ++i) {
+      const int lo = __shfl_sync(kFull, my_ptr, i);
+      const int hi = __shfl_sync(kFull, my_ptr, i + 1);
+      const int len = hi - lo;
+      if (len > a.heavy_threshold) {  // a heavy block writes this row: skip its indices
+        if (hi - b >= 32) {
+          const int nb = b + ((hi - b) & ~31);
+          if (nb == b + 32) { cur_u = nxt_u; cur_s = nxt_s; }
+          else load_batch<SCALED>(a, nb, stream_end, lane, cur_u, cur_s);
+          load_batch<SCALED>(a, (int64_t)nb + 32, stream_end, lane, nxt_u, nxt_s);
+          b = nb;
+        }
+        continue;
+      }
       V acc[CPL];
 #pragma unroll
       for (int c = 0; c < CPL; ++c) zero(acc[c]);
-      accumulate<VEC, G, CPL, SCALED>(a, lo, hi, 0, 1, f0, fend, acc);
+      int p = lo;
+      while (p < hi) {
+        if (p - b >= 32) {  // the stream is contiguous, so this is exactly one batch ahead
+          b += 32;
+          cur_u = nxt_u;
+          cur_s = nxt_s;
+          load_batch<SCALED>(a, (int64_t)b + 32, stream_end, lane, nxt_u, nxt_s);
+        }
+        const int e = min(hi - b, 32);
+        add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, p - b, e, grp, acc);
+        p = b + e;
+      }
+      combine_groups<VEC, G, CPL>(acc);
       if (lane < G) {
         const float rs = (a.mean_rows && len > 0) ? 1.0f / (float)len : 1.0f;
-        float* orow = a.Y + (size_t)r * (size_t)a.F;
+        float* orow = a.Y + (size_t)(rb + i) * (size_t)a.F + f0;
 #pragma unroll
         for (int c = 0; c < CPL; ++c) {
-          const int f = f0 + (c0 + c * G) * VEC;
-          if (f < fend) {
+          if (cok[c]) {
             if (a.mean_rows) scale(acc[c], rs);
-            stcs_vec(orow + f, acc[c]);
+            stcs_vec(orow + (c0 + c * G) * VEC, acc[c]);
           }
         }
       }
@@ -194,21 +257,32 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
     return;
   }
 
-  const int width = fend - f0;
   const int count = min(*a.heavy_count, a.heavy_cap);
   for (int i = blockIdx.x; i < count; i += heavy_blocks) {
     const int64_t r = a.heavy_list[i];
-    const int64_t lo = __ldg(a.ptr + r), hi = __ldg(a.ptr + r + 1);
+    const int lo = (int)__ldg(a.ptr + r), hi = (int)__ldg(a.ptr + r + 1);
     V acc[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) zero(acc[c]);
-    accumulate<VEC, G, CPL, SCALED>(a, lo, hi, warp, kWarpsPerBlock, f0, fend, acc);
+    // warp w sums batches w, w+8, ... of the segment
+    int32_t cur_u, nxt_u;
+    float cur_s, nxt_s;
+    int b = hi - lo > warp * 32 ? lo + warp * 32 : hi;
+    if (b < hi) load_batch<SCALED>(a, b, hi, lane, cur_u, cur_s);
+    while (b < hi) {
+      const bool more = hi - b > kBlock;
+      if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
+      add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
+      if (!more) break;
+      b += kBlock;
+      cur_u = nxt_u;
+      cur_s = nxt_s;
+    }
+    combine_groups<VEC, G, CPL>(acc);
     if (lane < G) {
 #pragma unroll
-      for (int c = 0; c < CPL; ++c) {
-        const int fl = (c0 + c * G) * VEC;
-        if (fl < width) st_smem(&part[warp][fl], acc[c]);
-      }
+      for (int c = 0; c < CPL; ++c)
+        if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
     }
     __syncthreads();
     const float rs = a.mean_rows ? 1.0f / (float)(hi - lo) : 1.0f;
@@ -227,7 +301,8 @@ template <int VEC, int G, int CPL, bool SCALED>
 dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
   if (a.n == 0) return DG_OK;
   const int heavy_blocks = g->sm_count * 2;
-  const int64_t blocks = heavy_blocks + (a.n + a.rows_per_block - 1) / a.rows_per_block;
+  const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
+  const int64_t blocks = heavy_blocks + (a.n + rows_per_block - 1) / rows_per_block;
   dim3 grid((unsigned)blocks, (unsigned)slices);
   ap_kernel<VEC, G, CPL, SCALED><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
   DG_CUDA(cudaGetLastError());

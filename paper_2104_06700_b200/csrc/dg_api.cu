@@ -54,10 +54,20 @@ static dg_status_t refresh_heavy(Graph* g, bool csr, bool csc, cudaStream_t s) {
   return DG_OK;
 }
 
+// rows_per_block is rounded up to a whole number of rows per warp (8 warps per block).
+static int32_t rows_per_warp(const Graph* g) {
+  int64_t r = (g->rows_per_block + 7) / 8;
+  return (int32_t)(r < 1 ? 1 : (r > 31 ? 31 : r));
+}
+
 static dg_status_t check_features(const Graph* g, const float* in, float* out, int32_t F,
                                   dg_op_t op) {
   if (!g) return invalid("graph handle is NULL");
   if (F < 1) return invalid("F must be >= 1");
+  if (F > (1 << 20)) {
+    set_error("F must be at most 2^20");
+    return DG_ERR_UNSUPPORTED;
+  }
   if (op != DG_OP_SUM && op != DG_OP_MEAN) return invalid("op must be DG_OP_SUM or DG_OP_MEAN");
   if (g->n > 0) {
     if (!in || !out) return invalid("feature matrix pointer is NULL");
@@ -201,7 +211,7 @@ dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op
   a.F = F;
   a.mean_rows = op == DG_OP_MEAN;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
-  a.rows_per_block = (int32_t)g->rows_per_block;
+  a.rows_per_warp = rows_per_warp(g);
   return aggregate_run(g, a, (cudaStream_t)stream);
 }
 
@@ -226,7 +236,7 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
   a.F = F;
   a.mean_rows = 0;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
-  a.rows_per_block = (int32_t)g->rows_per_block;
+  a.rows_per_warp = rows_per_warp(g);
   return aggregate_run(g, a, (cudaStream_t)stream);
 }
 
@@ -280,7 +290,7 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     return DG_OK;
   }
   if (!strcmp(name, "rows_per_block")) {
-    if (value < 1 || value > 4096) return invalid("rows_per_block must be in [1, 4096]");
+    if (value < 1 || value > 248) return invalid("rows_per_block must be in [1, 248]");
     g->rows_per_block = value;
     return DG_OK;
   }

@@ -58,7 +58,7 @@ struct ApArgs {
   int32_t slice_f;            // features per slice (multiple of the vector width)
   int32_t mean_rows;          // 1: multiply the finished row by 1/(segment length)
   int32_t heavy_threshold;
-  int32_t rows_per_block;
+  int32_t rows_per_warp;     // consecutive light segments per warp (1..31)
 };
 
 void set_error(const std::string& msg);
