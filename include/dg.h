@@ -81,7 +81,10 @@ dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t
  *   rowidx_T[q] destination vertex of edge perm[q] (int32)
  *   w_T[q]      edge_w[perm[q]], copied bit for bit (absent when the graph is unweighted)
  * There is exactly one correct result; it is integer work and bit-exact.
- *   csc_storage  device, 256-byte aligned, >= csc_bytes; holds the four arrays, is borrowed
+ * Next to these the storage holds two internal arrays: the per-edge factor w_T[q]/deg(rowidx_T[q])
+ * that the backward pass of the mean streams, and (for graphs with at least 64 edges per
+ * vertex) the split pointers of the CSC for source blocking.
+ *   csc_storage  device, 256-byte aligned, >= csc_bytes; holds all these arrays, is borrowed
  *                by the handle until destroy (or the next transpose) and is what
  *                dg_graph_get_csc points into
  *   scratch      device, 256-byte aligned, >= scratch_bytes; free for reuse once the work
@@ -143,6 +146,11 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
  *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows)
+ *   "l2_budget_mb"     MiB of the gathered matrix one launch may keep L2-resident
+ *   "source_blocks"    number of source-vertex ranges the pass is cut into, one launch each
+ *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,
+ *                      4, 8 or 16; ignored for graphs without split pointers, i.e. with fewer
+ *                      than 64 edges per vertex or unsorted rows)
  * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.
  */
 dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);

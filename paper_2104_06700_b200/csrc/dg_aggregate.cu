@@ -40,6 +40,13 @@ __device__ __forceinline__ float2 ldg_vec(const char* p, float2) {
 __device__ __forceinline__ float4 ldg_vec(const char* p, float4) {
   return __ldg(reinterpret_cast<const float4*>(p));
 }
+__device__ __forceinline__ float ld_vec(const float* p, float) { return *p; }
+__device__ __forceinline__ float2 ld_vec(const float* p, float2) {
+  return *reinterpret_cast<const float2*>(p);
+}
+__device__ __forceinline__ float4 ld_vec(const float* p, float4) {
+  return *reinterpret_cast<const float4*>(p);
+}
 __device__ __forceinline__ void zero(float& a) { a = 0.f; }
 __device__ __forceinline__ void zero(float2& a) { a.x = a.y = 0.f; }
 __device__ __forceinline__ void zero(float4& a) { a.x = a.y = a.z = a.w = 0.f; }
@@ -86,18 +93,17 @@ __device__ __forceinline__ void load_batch(const ApArgs& a, int64_t b, int end, 
   const int64_t k = b + lane;
   if (k < end) {
     u = __ldcs(a.idx + k);
-    if (SCALED) {
-      s = a.w ? __ldcs(a.w + k) : 1.f;
-      if (a.node_scale) s *= __ldg(a.node_scale + u);
-    }
+    if (SCALED) s = __ldcs(a.w + k);
   }
 }
 
 template <int VEC, int G, int CPL>
 struct Shape {
   static constexpr int NG = 32 / G;  // edges one warp-wide load instruction covers
-  static constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : 2);
-  static constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;  // load steps in flight per lane
+  // load steps in flight per lane (fewer when a step is several vectors wide), and no more
+  // steps than one 32-edge batch holds
+  static constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : (VEC <= 2 ? 4 : 2));
+  static constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;
 };
 
 // Adds the edges held in lanes [s, e) of the current batch (cur_u / cur_s: one edge per lane)
@@ -175,7 +181,7 @@ __device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL])
 // first, so the long segments start early); in the remaining blocks every warp owns
 // rows_per_warp consecutive light segments and streams their indices as one run of 32-edge
 // batches, the next batch always in flight while the current one is summed.
-template <int VEC, int G, int CPL, bool SCALED>
+template <int VEC, int G, int CPL, bool SCALED, bool SEG>
 __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
   using V = typename Vec<VEC>::T;
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
@@ -198,6 +204,85 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
     const int ci = c0 + c * G;
     cok[c] = ci < chunks;
     xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * 4u;
+  }
+
+  // Writes one finished row: scales by 1/length for the mean and, in a later source block, adds
+  // what the earlier blocks left in Y.
+  auto store_row = [&](int64_t r, int len, V (&acc)[CPL]) {
+    if (lane < G) {
+      const float rs = (a.mean_rows && len > 0) ? 1.0f / (float)len : 1.0f;
+      float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) {
+        if (cok[c]) {
+          float* dst = orow + (c0 + c * G) * VEC;
+          if (a.mean_rows) scale(acc[c], rs);
+          if (SEG && a.accumulate) add(acc[c], ld_vec(dst, V()));
+          stcs_vec(dst, acc[c]);
+        }
+      }
+    }
+  };
+
+  if (SEG && (int)blockIdx.x >= heavy_blocks) {
+    // Source-blocked pass: row i of this warp contributes the positions [seg_lo, seg_hi) of its
+    // segment.  The pieces are not adjacent in memory, so batches start at each piece; the
+    // prefetch cursor (qi, qb) runs one batch ahead of the summing loop across rows.
+    const int rpw = a.rows_per_warp;
+    const int64_t rb = ((int64_t)(blockIdx.x - heavy_blocks) * kWarpsPerBlock + warp) * rpw;
+    if (rb >= a.n) return;
+    const int nrows = (int)min((int64_t)rpw, a.n - rb);
+    int my_lo = 0, my_hi = 0, my_full = 0;
+    if (lane < nrows) {
+      my_lo = __ldg(a.seg_lo + rb + lane);
+      my_hi = __ldg(a.seg_hi + rb + lane);
+      my_full = (int)(__ldg(a.ptr + rb + lane + 1) - __ldg(a.ptr + rb + lane));
+    }
+    const unsigned heavy_mask = __ballot_sync(kFull, my_full > a.heavy_threshold);
+    const unsigned work =
+        __ballot_sync(kFull, lane < nrows && my_full <= a.heavy_threshold && my_hi > my_lo);
+    int qi = work ? __ffs(work) - 1 : 32, qb = 0, qhi = 0;
+    int32_t cur_u = 0, nxt_u = 0;
+    float cur_s = 0.f, nxt_s = 0.f;
+    auto step_q = [&]() {
+      qb += 32;
+      if (qb >= qhi) {
+        const unsigned rest = qi >= 31 ? 0u : (work & ~((2u << qi) - 1u));
+        qi = rest ? __ffs(rest) - 1 : 32;
+        if (qi < 32) {
+          qb = __shfl_sync(kFull, my_lo, qi);
+          qhi = __shfl_sync(kFull, my_hi, qi);
+        }
+      }
+    };
+    if (qi < 32) {
+      qb = __shfl_sync(kFull, my_lo, qi);
+      qhi = __shfl_sync(kFull, my_hi, qi);
+      load_batch<SCALED>(a, qb, qhi, lane, cur_u, cur_s);
+      step_q();
+      if (qi < 32) load_batch<SCALED>(a, qb, qhi, lane, nxt_u, nxt_s);
+    }
+    for (int i = 0; i < nrows; ++i) {
+      if ((heavy_mask >> i) & 1u) continue;
+      const int lo = __shfl_sync(kFull, my_lo, i);
+      const int hi = __shfl_sync(kFull, my_hi, i);
+      const int len = __shfl_sync(kFull, my_full, i);
+      V acc[CPL];
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) zero(acc[c]);
+      for (int b = lo; b < hi; b += 32) {
+        add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
+        cur_u = nxt_u;
+        cur_s = nxt_s;
+        if (qi < 32) {
+          step_q();
+          if (qi < 32) load_batch<SCALED>(a, qb, qhi, lane, nxt_u, nxt_s);
+        }
+      }
+      combine_groups<VEC, G, CPL>(acc);
+      store_row(rb + i, len, acc);
+    }
+    return;
   }
 
   if ((int)blockIdx.x >= heavy_blocks) {
@@ -242,17 +327,7 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
         p = b + e;
       }
       combine_groups<VEC, G, CPL>(acc);
-      if (lane < G) {
-        const float rs = (a.mean_rows && len > 0) ? 1.0f / (float)len : 1.0f;
-        float* orow = a.Y + (size_t)(rb + i) * (size_t)a.F + f0;
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          if (cok[c]) {
-            if (a.mean_rows) scale(acc[c], rs);
-            stcs_vec(orow + (c0 + c * G) * VEC, acc[c]);
-          }
-        }
-      }
+      store_row(rb + i, len, acc);
     }
     return;
   }
@@ -260,7 +335,9 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
   const int count = min(*a.heavy_count, a.heavy_cap);
   for (int i = blockIdx.x; i < count; i += heavy_blocks) {
     const int64_t r = a.heavy_list[i];
-    const int lo = (int)__ldg(a.ptr + r), hi = (int)__ldg(a.ptr + r + 1);
+    const int full = (int)(__ldg(a.ptr + r + 1) - __ldg(a.ptr + r));
+    const int lo = SEG ? __ldg(a.seg_lo + r) : (int)__ldg(a.ptr + r);
+    const int hi = SEG ? __ldg(a.seg_hi + r) : lo + full;
     V acc[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) zero(acc[c]);
@@ -285,13 +362,15 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
         if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
     }
     __syncthreads();
-    const float rs = a.mean_rows ? 1.0f / (float)(hi - lo) : 1.0f;
+    const float rs = a.mean_rows ? 1.0f / (float)full : 1.0f;
     float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
     for (int f = threadIdx.x; f < width; f += kBlock) {
       float t = part[0][f];
 #pragma unroll
       for (int w = 1; w < kWarpsPerBlock; ++w) t += part[w][f];
-      __stcs(orow + f, a.mean_rows ? t * rs : t);
+      if (a.mean_rows) t *= rs;
+      if (SEG && a.accumulate) t += orow[f];
+      __stcs(orow + f, t);
     }
     __syncthreads();
   }
@@ -304,7 +383,8 @@ dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
   const int64_t blocks = heavy_blocks + (a.n + rows_per_block - 1) / rows_per_block;
   dim3 grid((unsigned)blocks, (unsigned)slices);
-  ap_kernel<VEC, G, CPL, SCALED><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
+  if (a.seg_lo) ap_kernel<VEC, G, CPL, SCALED, true><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
+  else ap_kernel<VEC, G, CPL, SCALED, false><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
   DG_CUDA(cudaGetLastError());
   count_launches(1);
   return DG_OK;
@@ -324,28 +404,66 @@ dg_status_t dispatch_shape(const Graph* g, const ApArgs& a, int slices, cudaStre
 
 }  // namespace
 
-// Widest vector both matrices allow, then the slice width: at most 128 vectors per row slice
-// (4 per lane), narrowed until one slice of X fits the L2 budget so that repeated gathers of a
-// source row are served from L2 instead of HBM.
-dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, cudaStream_t s) {
+// Bytes of L2 one row slice of `slice` floats occupies: L2 allocates 128-byte lines, and a slice
+// that does not start on a line boundary in every row touches one more line.
+static double slice_footprint(int64_t F, int64_t slice) {
+  const int64_t bytes = slice * 4;
+  const bool aligned = (F * 4) % 128 == 0 && bytes % 128 == 0;
+  return (double)(((bytes + 127) / 128) * 128 + (aligned ? 0 : 128));
+}
+
+// Chooses the launch shape, then runs one launch per source block.
+//   vector width: the widest both matrices allow;
+//   slice: at most 128 vectors per row slice (4 per lane);
+//   source blocks (Algorithm 2 of the paper, with L2 in the role of the CPU cache): when one
+//     slice of X over all n rows exceeds the L2 budget and the segments carry split pointers,
+//     the neighbour ids are cut into 2, 4, 8 or 16 ranges and each range is a launch of its
+//     own, so that the rows of X a launch gathers stay L2-resident; later launches add to Y.
+//     Without split pointers the slice is narrowed instead (down to 32 floats).
+dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split, cudaStream_t s) {
   ApArgs a = a0;
+  if (a.n == 0) return DG_OK;
   const uintptr_t px = (uintptr_t)a.X, py = (uintptr_t)a.Y;
   int vec = 1;
   if (a.F % 4 == 0 && px % 16 == 0 && py % 16 == 0) vec = 4;
   else if (a.F % 2 == 0 && px % 8 == 0 && py % 8 == 0) vec = 2;
 
-  int64_t slice = g->slice_features;
-  if (slice <= 0) {
-    slice = a.F;
-    const double budget = 0.4 * (double)g->l2_bytes;
-    if ((double)a.n * a.F * 4.0 > budget) {
-      slice = (int64_t)(budget / ((double)a.n * 4.0));
-      if (slice < 32) slice = a.F;  // a slice under 128 bytes per row is not worth a pass
-    }
-  }
+  const double budget = (double)g->l2_budget_bytes;
+  const double avg_len = (double)g->nnz / (double)a.n;
   const int64_t cap = 128LL * vec;
+  int64_t slice = g->slice_features > 0 ? g->slice_features : (a.F < cap ? (int64_t)a.F : cap);
   if (slice > cap) slice = cap;
   if (slice > a.F) slice = a.F;
+  int nb = 1;
+  if (g->source_blocks > 0) {
+    nb = split ? (int)g->source_blocks : 1;
+  } else if (g->slice_features <= 0 && (double)a.n * slice_footprint(a.F, slice) > budget) {
+    if (split) {
+      // widest slice first; a candidate is feasible when some block count keeps one block of
+      // the slice inside the budget and leaves a row at least 32 edges per block on average
+      const int64_t widths[4] = {64LL * vec, 32LL * vec, 16LL * vec, 8LL * vec};
+      bool found = false;
+      for (int t = 0; t < 4 && !found; ++t) {
+        int64_t w = widths[t];
+        if (w > slice) w = slice;
+        int cand = 1;
+        while (cand < kFineBlocks && (double)a.n / cand * slice_footprint(a.F, w) > budget) cand *= 2;
+        if ((double)a.n / cand * slice_footprint(a.F, w) <= budget && avg_len / cand >= 32.0) {
+          slice = w;
+          nb = cand;
+          found = true;
+        }
+      }
+      if (!found) {  // as many blocks as the row length allows, narrowest slice
+        nb = 1;
+        while (nb < kFineBlocks && avg_len / (nb * 2) >= 32.0) nb *= 2;
+        if (slice > 8LL * vec) slice = 8LL * vec;
+      }
+    } else {
+      int64_t w = (int64_t)(budget / ((double)a.n * 4.0));
+      if (w >= 32) slice = w < slice ? w : slice;  // narrower than 128 bytes is not worth a pass
+    }
+  }
   slice = (slice / vec) * vec;
   if (slice < vec) slice = vec;
   // even out the slices: same count, smallest width that covers F
@@ -355,11 +473,22 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, cudaStream_t s) {
   if (even <= slice) slice = even;
   a.slice_f = (int32_t)slice;
   const int slices = (int)((a.F + slice - 1) / slice);
-  const bool scaled = a.w != nullptr || a.node_scale != nullptr;
+  const bool scaled = a.w != nullptr;
 
-  if (vec == 4) return scaled ? dispatch_shape<4, true>(g, a, slices, s) : dispatch_shape<4, false>(g, a, slices, s);
-  if (vec == 2) return scaled ? dispatch_shape<2, true>(g, a, slices, s) : dispatch_shape<2, false>(g, a, slices, s);
-  return scaled ? dispatch_shape<1, true>(g, a, slices, s) : dispatch_shape<1, false>(g, a, slices, s);
+  const int per = kFineBlocks / nb;
+  for (int j = 0; j < nb; ++j) {
+    if (nb > 1) {
+      a.seg_lo = split + (size_t)(j * per) * (size_t)a.n;
+      a.seg_hi = split + (size_t)((j + 1) * per) * (size_t)a.n;
+      a.accumulate = j > 0;
+    }
+    dg_status_t st;
+    if (vec == 4) st = scaled ? dispatch_shape<4, true>(g, a, slices, s) : dispatch_shape<4, false>(g, a, slices, s);
+    else if (vec == 2) st = scaled ? dispatch_shape<2, true>(g, a, slices, s) : dispatch_shape<2, false>(g, a, slices, s);
+    else st = scaled ? dispatch_shape<1, true>(g, a, slices, s) : dispatch_shape<1, false>(g, a, slices, s);
+    if (st != DG_OK) return st;
+  }
+  return DG_OK;
 }
 
 }  // namespace dg

@@ -35,6 +35,8 @@ static dg_status_t free_owned(Graph* g) {
   if (g->heavy_rows) cudaFree(g->heavy_rows);
   if (g->heavy_cols) cudaFree(g->heavy_cols);
   if (g->counters) cudaFree(g->counters);
+  if (g->split_csr) cudaFree(g->split_csr);
+  g->split_csr = nullptr;
   g->inv_deg = nullptr;
   g->heavy_rows = g->heavy_cols = g->counters = nullptr;
   return DG_OK;
@@ -109,6 +111,9 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (e != cudaSuccess) { delete g; return cuda_fail(e, "cudaGetDeviceProperties"); }
   g->sm_count = prop.multiProcessorCount;
   g->l2_bytes = (size_t)prop.l2CacheSize;
+  g->l2_budget_bytes = (int64_t)(g->l2_bytes * 3 / 10);
+  g->fine_rows = (n + kFineBlocks - 1) / kFineBlocks;
+  if (g->fine_rows < 1) g->fine_rows = 1;
   g->heavy_cap = nnz / 64 + 1;  // enough for any threshold >= 64
   if (g->heavy_cap > n) g->heavy_cap = n > 0 ? n : 1;
 
@@ -117,13 +122,23 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)g->heavy_cap * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->counters, 4 * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(g->counters, 0, 4 * sizeof(int32_t));
+  if (e == cudaSuccess && wants_split(n, nnz))
+    e = cudaMalloc(&g->split_csr, (size_t)(kFineBlocks + 1) * (size_t)n * sizeof(int32_t));
   if (e != cudaSuccess) { free_owned(g); delete g; return cuda_fail(e, "cudaMalloc (graph metadata)"); }
 
   dg_status_t st = build_degree_info(g, 0);
   if (st == DG_OK) st = refresh_heavy(g, true, false, 0);
+  if (st == DG_OK && g->split_csr)
+    st = build_split(rowptr, colidx, n, g->fine_rows, g->split_csr, g->counters + 3, 0);
   if (st == DG_OK) {
-    e = cudaStreamSynchronize(0);
+    int32_t unsorted = 0;
+    e = cudaMemcpy(&unsorted, g->counters + 3, sizeof(unsorted), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
     if (e != cudaSuccess) st = cuda_fail(e, "cudaStreamSynchronize (graph create)");
+    if (st == DG_OK && unsorted && g->split_csr) {  // rows not sorted: no source blocking
+      cudaFree(g->split_csr);
+      g->split_csr = nullptr;
+    }
   }
   if (st != DG_OK) { free_owned(g); delete g; return st; }
   *out_graph = g;
@@ -201,7 +216,6 @@ dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op
   a.ptr = g->rowptr;
   a.idx = g->colidx;
   a.w = g->edge_w;
-  a.node_scale = nullptr;
   a.X = H;
   a.Y = out;
   a.heavy_list = g->heavy_rows;
@@ -212,7 +226,7 @@ dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op
   a.mean_rows = op == DG_OP_MEAN;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, (cudaStream_t)stream);
+  return aggregate_run(g, a, g->split_csr, (cudaStream_t)stream);
 }
 
 dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t op, float* dH,
@@ -225,8 +239,7 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
   ApArgs a{};
   a.ptr = g->colptr;
   a.idx = g->rowidx_T;
-  a.w = g->w_T;
-  a.node_scale = op == DG_OP_MEAN ? g->inv_deg : nullptr;
+  a.w = op == DG_OP_MEAN ? g->mean_scale_T : g->w_T;
   a.X = dOut;
   a.Y = dH;
   a.heavy_list = g->heavy_cols;
@@ -237,7 +250,7 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
   a.mean_rows = 0;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, (cudaStream_t)stream);
+  return aggregate_run(g, a, g->split_csc, (cudaStream_t)stream);
 }
 
 size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F) {
@@ -294,6 +307,17 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     g->rows_per_block = value;
     return DG_OK;
   }
+  if (!strcmp(name, "l2_budget_mb")) {
+    if (value < 1 || value > 4096) return invalid("l2_budget_mb must be in [1, 4096]");
+    g->l2_budget_bytes = value << 20;
+    return DG_OK;
+  }
+  if (!strcmp(name, "source_blocks")) {
+    if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16)
+      return invalid("source_blocks must be 0 (automatic), 1, 2, 4, 8 or 16");
+    g->source_blocks = value;
+    return DG_OK;
+  }
   return invalid("unknown parameter name");
 }
 
@@ -302,6 +326,8 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
   if (!strcmp(name, "heavy_threshold")) { *value = g->heavy_threshold; return DG_OK; }
   if (!strcmp(name, "slice_features")) { *value = g->slice_features; return DG_OK; }
   if (!strcmp(name, "rows_per_block")) { *value = g->rows_per_block; return DG_OK; }
+  if (!strcmp(name, "l2_budget_mb")) { *value = g->l2_budget_bytes >> 20; return DG_OK; }
+  if (!strcmp(name, "source_blocks")) { *value = g->source_blocks; return DG_OK; }
   return invalid("unknown parameter name");
 }
 

@@ -52,6 +52,38 @@ __global__ void validate_colidx_kernel(const int32_t* __restrict__ colidx, int64
   if (bad) atomicOr(flags, 8);
 }
 
+// split[b * n + v] for b = 0..kFineBlocks: the first position of segment v whose id is
+// >= b * fine_rows, by binary search (the segment must be sorted ascending).
+__global__ void split_kernel(const int64_t* __restrict__ ptr, const int32_t* __restrict__ idx,
+                             int64_t n, int64_t fine_rows, int32_t* __restrict__ split) {
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= (int64_t)(kFineBlocks + 1) * n) return;
+  const int64_t b = t / n, v = t - b * n;
+  int64_t lo = ptr[v], hi = ptr[v + 1];
+  if (b == 0) { split[t] = (int32_t)lo; return; }
+  if (b == kFineBlocks) { split[t] = (int32_t)hi; return; }
+  const int64_t bound = b * fine_rows;
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(idx + mid) < bound) lo = mid + 1; else hi = mid;
+  }
+  split[t] = (int32_t)lo;
+}
+
+// One warp per segment: sets *flag when two adjacent ids of a segment are out of order.
+__global__ void sorted_check_kernel(const int64_t* __restrict__ ptr,
+                                    const int32_t* __restrict__ idx, int64_t n,
+                                    int32_t* __restrict__ flag) {
+  const int64_t v = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (v >= n) return;
+  const int lane = threadIdx.x & 31;
+  const int64_t lo = ptr[v], hi = ptr[v + 1];
+  int bad = 0;
+  for (int64_t k = lo + 1 + lane; k < hi; k += 32)
+    if (__ldg(idx + k - 1) > __ldg(idx + k)) bad = 1;
+  if (bad) atomicOr(flag, 1);
+}
+
 inline unsigned blocks_for(int64_t items) { return (unsigned)((items + kBlock - 1) / kBlock); }
 
 }  // namespace
@@ -71,6 +103,25 @@ dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, i
   heavy_list_kernel<<<blocks_for(n), kBlock, 0, s>>>(ptr, n, threshold, list, cap, count);
   DG_CUDA(cudaGetLastError());
   count_launches(1);
+  return DG_OK;
+}
+
+bool wants_split(int64_t n, int64_t nnz) {
+  return n >= 4096 && nnz >= kBlockingMinAvgLen * n &&
+         (int64_t)(kFineBlocks + 1) * n < ((int64_t)1 << 40);
+}
+
+// Fills the split pointers of one direction and raises *unsorted_flag (device) when a segment
+// is not sorted ascending, in which case the pointers must not be used.
+dg_status_t build_split(const int64_t* ptr, const int32_t* idx, int64_t n, int64_t fine_rows,
+                        int32_t* split, int32_t* unsorted_flag, cudaStream_t s) {
+  DG_CUDA(cudaMemsetAsync(unsorted_flag, 0, sizeof(int32_t), s));
+  sorted_check_kernel<<<blocks_for(n * 32), kBlock, 0, s>>>(ptr, idx, n, unsorted_flag);
+  DG_CUDA(cudaGetLastError());
+  split_kernel<<<blocks_for((int64_t)(kFineBlocks + 1) * n), kBlock, 0, s>>>(ptr, idx, n,
+                                                                            fine_rows, split);
+  DG_CUDA(cudaGetLastError());
+  count_launches(2);
   return DG_OK;
 }
 

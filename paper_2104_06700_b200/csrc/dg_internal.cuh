@@ -16,17 +16,26 @@ struct dg_graph {
   const int32_t* colidx = nullptr;
   const float* edge_w = nullptr;
 
-  float* inv_deg = nullptr;      // n: 1/deg(v), 0 for empty rows (mean backward gathers it)
+  float* inv_deg = nullptr;      // n: 1/deg(v), 0 for empty rows (the transpose folds it into mean_scale_T)
   int32_t* heavy_rows = nullptr; // CSR rows longer than heavy_threshold (forward)
   int32_t* heavy_cols = nullptr; // CSC columns longer than heavy_threshold (backward)
   int32_t* counters = nullptr;   // [0] #heavy rows, [1] #heavy cols, [2] validation flags
   int64_t heavy_cap = 0;         // capacity of each heavy list
+
+  // Source blocking: the neighbour ids are cut into kFineBlocks ranges of fine_rows ids;
+  // split[b * n + v] is the first position of segment v whose neighbour id is >= b * fine_rows
+  // (entry kFineBlocks is the segment end).  Built only for graphs whose rows are long and
+  // sorted; nullptr otherwise.  split_csr is owned, split_csc lives in the caller's CSC storage.
+  int32_t* split_csr = nullptr;
+  int32_t* split_csc = nullptr;
+  int64_t fine_rows = 0;
 
   bool transposed = false;
   const int64_t* colptr = nullptr;
   const int32_t* rowidx_T = nullptr;
   const float* w_T = nullptr;
   const int32_t* perm = nullptr;
+  const float* mean_scale_T = nullptr;  // w_T[q] / deg(rowidx_T[q]): edge factor of the mean's backward
 
   int device = 0;
   int sm_count = 148;
@@ -35,19 +44,23 @@ struct dg_graph {
   int64_t heavy_built_for = 0;   // threshold the heavy lists were built with
   int64_t slice_features = 0;    // 0 = automatic
   int64_t rows_per_block = 32;
+  int64_t l2_budget_bytes = 0;   // bytes of the gathered matrix one launch may keep L2-resident
+  int64_t source_blocks = 0;     // 0 = automatic, else 1, 2, 4, 8 or 16
 };
 
 namespace dg {
 
 using Graph = ::dg_graph;
 
+constexpr int kFineBlocks = 16;          // finest cut of the neighbour ids for source blocking
+constexpr int64_t kBlockingMinAvgLen = 64;  // split pointers are built when nnz >= 64 n
+
 // One direction of AP as the kernels see it: out[r] = rs_r * sum_k s_k * X[idx[k]],
-// s_k = w[k] * node_scale[idx[k]] (either factor may be absent).
+// s_k = w[k] (1 when w is absent).
 struct ApArgs {
   const int64_t* ptr;         // n+1 segment pointers (rowptr or colptr)
   const int32_t* idx;         // neighbour ids (colidx or rowidx_T)
   const float* w;             // per-edge weight or nullptr
-  const float* node_scale;    // per-neighbour factor (1/deg) or nullptr
   const float* X;             // n x F input
   float* Y;                   // n x F output
   const int32_t* heavy_list;  // segments longer than heavy_threshold
@@ -59,6 +72,9 @@ struct ApArgs {
   int32_t mean_rows;          // 1: multiply the finished row by 1/(segment length)
   int32_t heavy_threshold;
   int32_t rows_per_warp;     // consecutive light segments per warp (1..31)
+  const int32_t* seg_lo;      // source-blocked pass: first and one-past-last position of every
+  const int32_t* seg_hi;      //   segment's piece (n entries each); nullptr = whole segments
+  int32_t accumulate;         // source-blocked pass after the first: add to what Y holds
 };
 
 void set_error(const std::string& msg);
@@ -76,6 +92,9 @@ dg_status_t build_degree_info(Graph* g, cudaStream_t s);
 dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, int32_t* list,
                              int64_t cap, int32_t* count, cudaStream_t s);
 dg_status_t validate_csr(Graph* g, cudaStream_t s, int* flags_host);
+bool wants_split(int64_t n, int64_t nnz);
+dg_status_t build_split(const int64_t* ptr, const int32_t* idx, int64_t n, int64_t fine_rows,
+                        int32_t* split, int32_t* unsorted_flag, cudaStream_t s);
 
 // dg_transpose.cu
 void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
@@ -83,6 +102,6 @@ void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
 dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s);
 
 // dg_aggregate.cu
-dg_status_t aggregate_run(const Graph* g, const ApArgs& a, cudaStream_t s);
+dg_status_t aggregate_run(const Graph* g, const ApArgs& a, const int32_t* split, cudaStream_t s);
 
 }  // namespace dg

@@ -219,11 +219,15 @@ __global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int
   for (int64_t u = prev + 1; u <= cur; ++u) colptr[u] = q;
 }
 
-// rowidx_T[q] = the row r with rowptr[r] <= perm[q] < rowptr[r+1];  w_T[q] = edge_w[perm[q]].
+// rowidx_T[q] = the row r with rowptr[r] <= perm[q] < rowptr[r+1];  w_T[q] = edge_w[perm[q]];
+// mean_scale_T[q] = w_T[q] (1 if unweighted) / deg(r), the factor of edge q in the backward
+// pass of the mean, so that the backward kernel streams it instead of gathering 1/deg.
 __global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64_t nnz,
                                         const int64_t* __restrict__ rowptr, int64_t n,
                                         const float* __restrict__ edge_w,
-                                        int32_t* __restrict__ rowidx_T, float* __restrict__ w_T) {
+                                        const float* __restrict__ inv_deg,
+                                        int32_t* __restrict__ rowidx_T, float* __restrict__ w_T,
+                                        float* __restrict__ mean_scale_T) {
   const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (q >= nnz) return;
   const int64_t k = perm[q];
@@ -233,14 +237,19 @@ __global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64
     if (__ldg(rowptr + mid) <= k) lo = mid; else hi = mid;
   }
   rowidx_T[q] = (int32_t)lo;
-  if (edge_w) w_T[q] = edge_w[k];
+  float w = 1.f;
+  if (edge_w) {
+    w = edge_w[k];
+    w_T[q] = w;
+  }
+  mean_scale_T[q] = w * __ldg(inv_deg + lo);
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Layout {
   // csc storage
-  size_t colptr_off, rowidx_off, perm_off, w_off, csc_bytes;
+  size_t colptr_off, rowidx_off, perm_off, w_off, mscale_off, split_off, csc_bytes;
   // scratch
   size_t keys_a_off, keys_b_off, vals_off, hist_off, sums_off, scratch_bytes;
   int64_t tiles, hist_len, chunks;
@@ -254,6 +263,8 @@ Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
   L.rowidx_off = o; o += align256((size_t)nnz * 4);
   L.perm_off = o;   o += align256((size_t)nnz * 4);
   L.w_off = o;      o += weighted ? align256((size_t)nnz * 4) : 0;
+  L.mscale_off = o; o += align256((size_t)nnz * 4);
+  L.split_off = o;  o += wants_split(n, nnz) ? align256((size_t)(kFineBlocks + 1) * n * 4) : 0;
   L.csc_bytes = o > 0 ? o : 256;
   int bits = 1;
   while (bits < 31 && ((int64_t)1 << bits) < n) ++bits;
@@ -290,6 +301,7 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
   int32_t* rowidx_T = reinterpret_cast<int32_t*>(cb + L.rowidx_off);
   uint32_t* perm = reinterpret_cast<uint32_t*>(cb + L.perm_off);
   float* w_T = weighted ? reinterpret_cast<float*>(cb + L.w_off) : nullptr;
+  float* mean_scale_T = reinterpret_cast<float*>(cb + L.mscale_off);
   uint32_t* keys_buf[2] = {reinterpret_cast<uint32_t*>(sb + L.keys_a_off),
                            reinterpret_cast<uint32_t*>(sb + L.keys_b_off)};
   uint32_t* vals_tmp = reinterpret_cast<uint32_t*>(sb + L.vals_off);
@@ -325,7 +337,8 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
     colptr_from_sorted_keys<<<b1, 256, 0, s>>>(keys_in, nnz, n, colptr);
     DG_CUDA(cudaGetLastError());
     const unsigned b2 = (unsigned)((nnz + 255) / 256);
-    gather_rows_and_weights<<<b2, 256, 0, s>>>(perm, nnz, g->rowptr, n, g->edge_w, rowidx_T, w_T);
+    gather_rows_and_weights<<<b2, 256, 0, s>>>(perm, nnz, g->rowptr, n, g->edge_w, g->inv_deg,
+                                               rowidx_T, w_T, mean_scale_T);
     DG_CUDA(cudaGetLastError());
     count_launches(2);
   }
@@ -333,6 +346,15 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
   g->rowidx_T = rowidx_T;
   g->perm = reinterpret_cast<const int32_t*>(perm);
   g->w_T = w_T;
+  g->mean_scale_T = mean_scale_T;
+  g->split_csc = nullptr;
+  if (wants_split(n, nnz)) {
+    // the columns come out of the stable sort ordered by row, so the check never fires here
+    int32_t* split = reinterpret_cast<int32_t*>(cb + L.split_off);
+    if (dg_status_t st = build_split(colptr, rowidx_T, n, g->fine_rows, split, g->counters + 3, s))
+      return st;
+    g->split_csc = split;
+  }
   return DG_OK;
 }
 

@@ -178,6 +178,50 @@ def test_unsorted_rows_duplicates_and_self_loops():
     check_fwd_bwd(g, (rowptr, src, w), H, G, binding.DG_OP_MEAN, csc)
 
 
+# ------------------------------------------------------------------ source blocking
+@pytest.mark.parametrize("blocks,budget_mb", [(2, 31), (4, 31), (16, 31), (0, 1), (0, 2)])
+def test_source_blocked_passes_match_the_oracle(blocks, budget_mb):
+    """A graph with >= 64 edges per vertex carries split pointers; cutting the source ids into
+    2..16 ranges (one launch each, later launches adding to the output) must not change the
+    result beyond the summation order.  blocks = 0 lets a small L2 budget choose the cut."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.02)
+    assert sg.nnz >= 64 * sg.n
+    g = make_graph(sg)
+    g.dg_graph_set_param("source_blocks", blocks)
+    g.dg_graph_set_param("l2_budget_mb", budget_mb)
+    g.dg_graph_set_param("heavy_threshold", 256)      # some rows take the block-per-row path
+    csc = check_transpose(g, *host_csr(sg))
+    for F in (602, 64, 100, 7):
+        H = synth.features(sg.n, F, 41, DEV)
+        G = synth.features(sg.n, F, 42, DEV)
+        for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+            check_fwd_bwd(g, host_csr(sg), H, G, op, csc)
+
+
+def test_source_blocking_weighted_and_unsorted_rows():
+    """Weighted dense-ish graph; then the same edges with every row shuffled: the CSR loses its
+    split pointers (rows unsorted) while the CSC, sorted by construction, keeps them."""
+    rng = np.random.default_rng(5)
+    n, deg, F = 5000, 80, 48
+    src = np.stack([np.sort(rng.choice(n, deg, replace=False)) for _ in range(n)]).astype(np.int32)
+    rowptr = np.arange(n + 1, dtype=np.int64) * deg
+    w = rng.random(n * deg).astype(np.float32)
+    H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
+    for shuffle in (False, True):
+        cols = src.copy()
+        if shuffle:
+            for v in range(n):
+                rng.shuffle(cols[v])
+        cols = cols.reshape(-1)
+        g = binding.dg_graph_create(n, n * deg, torch.as_tensor(rowptr, device=DEV),
+                                    torch.as_tensor(cols, device=DEV),
+                                    torch.as_tensor(w, device=DEV))
+        g.dg_graph_set_param("source_blocks", 8)
+        csc = check_transpose(g, rowptr, cols, w)
+        for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+            check_fwd_bwd(g, (rowptr, cols, w), H, G, op, csc)
+
+
 # ------------------------------------------------------------------ errors never trap
 def test_error_statuses(tiny):
     g = make_graph(tiny)
