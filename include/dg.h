@@ -94,6 +94,32 @@ dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t
 dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes,
                                void* scratch, size_t scratch_bytes, void* stream);
 
+/*
+ * (The paper has no counterpart of this entry point; it exists for deployment reasons.)
+ * dg_graph_transpose for callers that cannot provide scratch memory: a plug-in inside a host
+ * program that has claimed the whole device for its own pool, a serving loop that must not hit
+ * the device-wide synchronisation of cudaMalloc/cudaFree, an embedder that owns nothing but the
+ * arrays it was handed.  The sort's scratch lives in an array of
+ * DG_TRANSPOSE_STATIC_SCRATCH_BYTES bytes inside the library image: every GPU on which the
+ * process loads the library holds that much from load to exit.  The call allocates and frees
+ * nothing, neither directly nor through a library.
+ *   - Same result, arguments and errors as dg_graph_transpose (csc_storage is still the
+ *     caller's: it is an output), minus the scratch pair.
+ *   - Limit: graphs whose scratch_bytes (dg_graph_transpose_workspace) exceed the array are
+ *     rejected with DG_ERR_UNSUPPORTED and a message that states both sizes; that is a little
+ *     under 1.4 million edges.
+ *   - The first call on a device looks up the array's device address (the device must be
+ *     current; the result is cached per device).  Make that first call before any stream
+ *     capture begins.
+ *   - All calls of a process on one device share the one array.  It keeps whatever the last
+ *     call left, which is harmless (every part is rewritten before it is read), but two calls
+ *     whose work overlaps on the GPU (different streams, or different threads) race on it and
+ *     give wrong CSC arrays: serialise them.
+ */
+#define DG_TRANSPOSE_STATIC_SCRATCH_BYTES (16u << 20)
+dg_status_t dg_graph_transpose_static(dg_graph_t g, void* csc_storage, size_t csc_bytes,
+                                      void* stream);
+
 /* Device pointers to the CSC arrays inside csc_storage (any output pointer may be NULL).
  * *w_T is set to NULL for an unweighted graph. */
 dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t** rowidx_T,

@@ -25,7 +25,7 @@ DG_OP_MEAN = 1
 
 EXPORTS = [
     "dg_graph_create", "dg_graph_destroy", "dg_graph_validate", "dg_graph_transpose_workspace",
-    "dg_graph_transpose", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
+    "dg_graph_transpose", "dg_graph_transpose_static", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
     "dg_aggregate_host_workspace", "dg_aggregate_host", "dg_graph_set_param",
     "dg_graph_get_param", "dg_kernel_launch_count", "dg_last_error", "dg_version",
 ]
@@ -57,6 +57,7 @@ def lib() -> ctypes.CDLL:
         L.dg_graph_validate.argtypes = [p, p]
         L.dg_graph_transpose_workspace.argtypes = [p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.dg_graph_transpose.argtypes = [p, p, sz, p, sz, p]
+        L.dg_graph_transpose_static.argtypes = [p, p, sz, p]
         L.dg_graph_get_csc.argtypes = [p, pp, pp, pp, pp]
         L.dg_aggregate_fwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_bwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
@@ -167,6 +168,19 @@ class Graph:
             ctypes.c_void_p(scratch.data_ptr()), scratch.numel(), _stream(stream)))
         self._csc = csc_storage
         scratch.record_stream(torch.cuda.current_stream() if stream is None else stream)
+
+    def dg_graph_transpose_static(self, csc_storage: Optional[torch.Tensor] = None,
+                                  stream=None) -> None:
+        """Builds the CSC with the scratch that is built into the library (small graphs only;
+        larger ones raise DgError with status DG_ERR_UNSUPPORTED).  Only the output storage is
+        a torch tensor; the call itself allocates nothing when that tensor is passed in."""
+        need_csc, _ = self.dg_graph_transpose_workspace()
+        if csc_storage is None:
+            csc_storage = torch.empty(need_csc, dtype=torch.uint8, device=self.device)
+        _check(lib().dg_graph_transpose_static(
+            self._h, ctypes.c_void_p(csc_storage.data_ptr()), csc_storage.numel(),
+            _stream(stream)))
+        self._csc = csc_storage
 
     def dg_graph_get_csc(self):
         """(colptr int64[n+1], rowidx_T int32[nnz], w_T fp32[nnz] | None, perm int32[nnz]) as
