@@ -173,6 +173,10 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
  *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows)
  *   "l2_budget_mb"     MiB of the gathered matrix one launch may keep L2-resident
+ *   "flat_rows"        kernel whose load steps run over row boundaries, for short rows:
+ *                      -1 = when rows average under 128 edges and no source blocking applies,
+ *                      0 = never, 1 = always (without source blocking)
+ *   "flat_rows_per_warp"  rows per warp of that kernel (0 = about 256 edges per warp, else 1..31)
  *   "source_blocks"    number of source-vertex ranges the pass is cut into, one launch each
  *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,
  *                      4, 8 or 16; ignored for graphs without split pointers, i.e. with fewer

@@ -312,6 +312,16 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     g->l2_budget_bytes = value << 20;
     return DG_OK;
   }
+  if (!strcmp(name, "flat_rows")) {
+    if (value < -1 || value > 1) return invalid("flat_rows must be -1 (automatic), 0 or 1");
+    g->flat_rows = value;
+    return DG_OK;
+  }
+  if (!strcmp(name, "flat_rows_per_warp")) {
+    if (value < 0 || value > 31) return invalid("flat_rows_per_warp must be in [0, 31]");
+    g->flat_rows_per_warp = value;
+    return DG_OK;
+  }
   if (!strcmp(name, "source_blocks")) {
     if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16)
       return invalid("source_blocks must be 0 (automatic), 1, 2, 4, 8 or 16");
@@ -328,6 +338,8 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
   if (!strcmp(name, "rows_per_block")) { *value = g->rows_per_block; return DG_OK; }
   if (!strcmp(name, "l2_budget_mb")) { *value = g->l2_budget_bytes >> 20; return DG_OK; }
   if (!strcmp(name, "source_blocks")) { *value = g->source_blocks; return DG_OK; }
+  if (!strcmp(name, "flat_rows")) { *value = g->flat_rows; return DG_OK; }
+  if (!strcmp(name, "flat_rows_per_warp")) { *value = g->flat_rows_per_warp; return DG_OK; }
   return invalid("unknown parameter name");
 }
 

@@ -49,9 +49,14 @@ def test_tiny_transpose_bit_exact(tiny, weighted):
 @pytest.mark.parametrize("F", [64, 8, 100, 602, 256, 128, 1, 3, 6, 130, 1028])
 @pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
 @pytest.mark.parametrize("weighted", [True, False])
-def test_tiny_forward_backward(tiny, F, op, weighted):
+@pytest.mark.parametrize("flat", [0, 1])
+def test_tiny_forward_backward(tiny, F, op, weighted, flat):
+    """flat = 1: the kernel whose load steps run over row boundaries (what short rows get by
+    default); flat = 0: the row-by-row kernel."""
     sg = tiny if weighted else synth.make("tiny", weighted=False)
     g = make_graph(sg)
+    g.dg_graph_set_param("flat_rows", flat)
+    g.dg_graph_set_param("heavy_threshold", 256)
     csc = check_transpose(g, *host_csr(sg))
     H = synth.features(sg.n, F, 100 + F, DEV)
     G = synth.features(sg.n, F, 200 + F, DEV)
@@ -80,10 +85,13 @@ def test_tiny_launch_shapes(tiny, slice_f, heavy, rows_per_block):
     g.dg_graph_set_param("rows_per_block", rows_per_block)
     assert g.dg_graph_get_param("heavy_threshold") == heavy
     csc = check_transpose(g, *host_csr(tiny))
-    for F in (64, 602, 10):
-        H = synth.features(tiny.n, F, 5, DEV)
-        G = synth.features(tiny.n, F, 6, DEV)
-        check_fwd_bwd(g, host_csr(tiny), H, G, binding.DG_OP_MEAN, csc)
+    for flat, rpw in ((0, 0), (1, 0), (1, 1), (1, 31)):
+        g.dg_graph_set_param("flat_rows", flat)
+        g.dg_graph_set_param("flat_rows_per_warp", rpw)
+        for F in (64, 602, 10):
+            H = synth.features(tiny.n, F, 5, DEV)
+            G = synth.features(tiny.n, F, 6, DEV)
+            check_fwd_bwd(g, host_csr(tiny), H, G, binding.DG_OP_MEAN, csc)
 
 
 def test_unaligned_feature_pointers(tiny):
@@ -119,13 +127,15 @@ def test_identity_and_ring_bit_exact():
 
 
 @pytest.mark.parametrize("F", [8, 100, 602])
-def test_star_graph_heavy_row_and_column(F):
+@pytest.mark.parametrize("flat", [0, 1])
+def test_star_graph_heavy_row_and_column(F, flat):
     """Vertex 0 pulls from every other vertex (one CSR row of n-1 entries, a heavy row), and
     every other vertex pulls from vertex 1 (one CSC column of n-1 entries)."""
     n = 6000
     rows = [list(range(1, n))] + [[1] for _ in range(n - 1)]
     w = np.random.default_rng(0).random(2 * (n - 1)).astype(np.float32)
     g, rowptr, colidx = csr_graph(n, rows, weights=w)
+    g.dg_graph_set_param("flat_rows", flat)
     csc = check_transpose(g, rowptr, colidx, w)
     H = synth.features(n, F, 11, DEV)
     G = synth.features(n, F, 12, DEV)
@@ -176,6 +186,24 @@ def test_unsorted_rows_duplicates_and_self_loops():
     csc = check_transpose(g, rowptr, src, w)
     H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
     check_fwd_bwd(g, (rowptr, src, w), H, G, binding.DG_OP_MEAN, csc)
+
+
+# ------------------------------------------------------------------ flat-stream kernel
+def test_flat_kernel_empty_rows_and_deterministic_bits():
+    """Rows of 0..39 edges, every third row empty: runs of empty rows inside and at the end of a
+    warp's stream; the same call twice gives the same bits."""
+    n, F = 3000, 64
+    rng = np.random.default_rng(3)
+    rows = [sorted(rng.choice(n, rng.integers(0, 40), replace=False).tolist()) if v % 3 else []
+            for v in range(n)]
+    g, rowptr, colidx = csr_graph(n, rows)
+    g.dg_graph_set_param("flat_rows", 1)
+    csc = check_transpose(g, rowptr, colidx, None)
+    for F in (64, 20, 200):
+        H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
+        check_fwd_bwd(g, (rowptr, colidx, None), H, G, binding.DG_OP_MEAN, csc)
+    a = g.dg_aggregate_fwd(H, binding.DG_OP_SUM).clone()
+    assert torch.equal(a, g.dg_aggregate_fwd(H, binding.DG_OP_SUM))
 
 
 # ------------------------------------------------------------------ source blocking
