@@ -169,14 +169,12 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
 /*
  * Tuning knobs (defaults come from the device's L2 size and SM count):
  *   "heavy_threshold"  rows longer than this are summed by a whole thread block
+ *   "heavy_blocks_per_sm"  thread blocks per SM that walk the list of heavy rows (longest first)
+ *                      before the launch turns to the light rows; 0 = as many as are resident
  *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
  *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows)
  *   "l2_budget_mb"     MiB of the gathered matrix one launch may keep L2-resident
- *   "flat_rows"        kernel whose load steps run over row boundaries, for short rows:
- *                      -1 = when rows average under 128 edges and no source blocking applies,
- *                      0 = never, 1 = always (without source blocking)
- *   "flat_rows_per_warp"  rows per warp of that kernel (0 = about 256 edges per warp, else 1..31)
  *   "source_blocks"    number of source-vertex ranges the pass is cut into, one launch each
  *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,
  *                      4, 8 or 16; ignored for graphs without split pointers, i.e. with fewer

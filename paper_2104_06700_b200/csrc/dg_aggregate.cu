@@ -97,12 +97,15 @@ __device__ __forceinline__ void load_batch(const ApArgs& a, int64_t b, int end, 
   }
 }
 
+#ifndef DG_U_CPL1
+#define DG_U_CPL1 8
+#endif
 template <int VEC, int G, int CPL>
 struct Shape {
   static constexpr int NG = 32 / G;  // edges one warp-wide load instruction covers
   // load steps in flight per lane (fewer when a step is several vectors wide), and no more
   // steps than one 32-edge batch holds
-  static constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : (VEC <= 2 ? 4 : 2));
+  static constexpr int U0 = CPL == 1 ? DG_U_CPL1 : (CPL == 2 ? 4 : (VEC <= 2 ? 4 : 2));
   static constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;
 };
 
@@ -118,49 +121,54 @@ __device__ __forceinline__ void add_edges(const char* const (&xrow)[CPL], uint32
   constexpr int NG = Shape<VEC, G, CPL>::NG;
   constexpr int U = Shape<VEC, G, CPL>::U;
   int p = s;
+  // With one vector per lane (8 steps in flight) the edge factors are fetched while adding, so
+  // that they hold no registers during the loads: that regime lives on occupancy.  With wider
+  // lanes (4 or 2 steps) they are fetched with the loads and the adds do not wait for a shuffle.
+  constexpr bool kLate = CPL == 1;
   for (; p + U * NG <= e; p += U * NG) {
     V v[U][CPL];
-    float sc[U];
+    float sc[kLate ? 1 : U];
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       const int src = p + j * NG + grp;
       const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src);
-      if (SCALED) sc[j] = __shfl_sync(kFull, cur_s, src);
+      if (SCALED && !kLate) sc[j] = __shfl_sync(kFull, cur_s, src);
       const uint64_t off = (uint64_t)u * row_bytes;
 #pragma unroll
       for (int c = 0; c < CPL; ++c) v[j][c] = ldg_vec(xrow[c] + off, V());
     }
 #pragma unroll
     for (int j = 0; j < U; ++j) {
+      float sj = 1.f;
+      if (SCALED) sj = kLate ? __shfl_sync(kFull, cur_s, p + j * NG + grp) : sc[j];
 #pragma unroll
       for (int c = 0; c < CPL; ++c) {
-        if (SCALED) fma(acc[c], sc[j], v[j][c]);
+        if (SCALED) fma(acc[c], sj, v[j][c]);
         else add(acc[c], v[j][c]);
       }
     }
   }
   if (p < e) {
     V v[U][CPL];
-    float sc[U];
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       const int src = p + j * NG + grp;
-      const bool ok = src < e;
       const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src & 31);
-      sc[j] = SCALED ? __shfl_sync(kFull, cur_s, src & 31) : 1.f;
-      if (!ok) sc[j] = 0.f;
       const uint64_t off = (uint64_t)u * row_bytes;
 #pragma unroll
       for (int c = 0; c < CPL; ++c) {
-        if (ok) v[j][c] = ldg_vec(xrow[c] + off, V());
-        else zero(v[j][c]);
+        if (src < e) v[j][c] = ldg_vec(xrow[c] + off, V());
+        else zero(v[j][c]);  // an absent edge adds zeros (times whatever factor its lane holds)
       }
     }
 #pragma unroll
     for (int j = 0; j < U; ++j) {
+      const int src = p + j * NG + grp;
+      float sj = SCALED ? __shfl_sync(kFull, cur_s, src & 31) : 1.f;
+      if (SCALED && src >= e) sj = 0.f;  // lanes past the batch hold neutral factors, not NaNs
 #pragma unroll
       for (int c = 0; c < CPL; ++c) {
-        if (SCALED) fma(acc[c], sc[j], v[j][c]);
+        if (SCALED) fma(acc[c], sj, v[j][c]);
         else add(acc[c], v[j][c]);
       }
     }
@@ -174,6 +182,73 @@ __device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL])
   for (int off = G; off < 32; off <<= 1) {
 #pragma unroll
     for (int c = 0; c < CPL; ++c) add(acc[c], shfl_xor(acc[c], off));
+  }
+}
+
+// Block-per-row path for the heavy segments: block x of the first `heavy_blocks` blocks takes
+// entries x, x + heavy_blocks, ... of the heavy list; its 8 warps sum interleaved 32-edge
+// batches and the partial sums are combined in shared memory in warp order.
+template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+__device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_blocks,
+                                           float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
+  using V = typename Vec<VEC>::T;
+  const int lane = threadIdx.x & 31;
+  const int warp = threadIdx.x >> 5;
+  const int grp = lane / G;
+  const int c0 = lane % G;
+  const int f0 = blockIdx.y * a.slice_f;
+  const int width = min(a.F, f0 + a.slice_f) - f0;
+  const int chunks = width / VEC;
+  const uint32_t row_bytes = (uint32_t)a.F * 4u;
+  const char* xrow[CPL];
+  bool cok[CPL];
+#pragma unroll
+  for (int c = 0; c < CPL; ++c) {
+    const int ci = c0 + c * G;
+    cok[c] = ci < chunks;
+    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * 4u;
+  }
+  const int count = min(*a.heavy_count, a.heavy_cap);
+  for (int i = blockIdx.x; i < count; i += heavy_blocks) {
+    const int64_t r = a.heavy_list[i];
+    const int full = (int)(__ldg(a.ptr + r + 1) - __ldg(a.ptr + r));
+    const int lo = SEG ? __ldg(a.seg_lo + r) : (int)__ldg(a.ptr + r);
+    const int hi = SEG ? __ldg(a.seg_hi + r) : lo + full;
+    V acc[CPL];
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) zero(acc[c]);
+    // warp w sums batches w, w+8, ... of the segment
+    int32_t cur_u, nxt_u;
+    float cur_s, nxt_s;
+    int b = hi - lo > warp * 32 ? lo + warp * 32 : hi;
+    if (b < hi) load_batch<SCALED>(a, b, hi, lane, cur_u, cur_s);
+    while (b < hi) {
+      const bool more = hi - b > kBlock;
+      if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
+      add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
+      if (!more) break;
+      b += kBlock;
+      cur_u = nxt_u;
+      cur_s = nxt_s;
+    }
+    combine_groups<VEC, G, CPL>(acc);
+    if (lane < G) {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c)
+        if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
+    }
+    __syncthreads();
+    const float rs = a.mean_rows ? 1.0f / (float)full : 1.0f;
+    float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
+    for (int f = threadIdx.x; f < width; f += kBlock) {
+      float t = part[0][f];
+#pragma unroll
+      for (int w = 1; w < kWarpsPerBlock; ++w) t += part[w][f];
+      if (a.mean_rows) t *= rs;
+      if (SEG && a.accumulate) t += orow[f];
+      __stcs(orow + f, t);
+    }
+    __syncthreads();
   }
 }
 
@@ -332,188 +407,30 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
     return;
   }
 
-  const int count = min(*a.heavy_count, a.heavy_cap);
-  for (int i = blockIdx.x; i < count; i += heavy_blocks) {
-    const int64_t r = a.heavy_list[i];
-    const int full = (int)(__ldg(a.ptr + r + 1) - __ldg(a.ptr + r));
-    const int lo = SEG ? __ldg(a.seg_lo + r) : (int)__ldg(a.ptr + r);
-    const int hi = SEG ? __ldg(a.seg_hi + r) : lo + full;
-    V acc[CPL];
-#pragma unroll
-    for (int c = 0; c < CPL; ++c) zero(acc[c]);
-    // warp w sums batches w, w+8, ... of the segment
-    int32_t cur_u, nxt_u;
-    float cur_s, nxt_s;
-    int b = hi - lo > warp * 32 ? lo + warp * 32 : hi;
-    if (b < hi) load_batch<SCALED>(a, b, hi, lane, cur_u, cur_s);
-    while (b < hi) {
-      const bool more = hi - b > kBlock;
-      if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
-      add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
-      if (!more) break;
-      b += kBlock;
-      cur_u = nxt_u;
-      cur_s = nxt_s;
-    }
-    combine_groups<VEC, G, CPL>(acc);
-    if (lane < G) {
-#pragma unroll
-      for (int c = 0; c < CPL; ++c)
-        if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
-    }
-    __syncthreads();
-    const float rs = a.mean_rows ? 1.0f / (float)full : 1.0f;
-    float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
-    for (int f = threadIdx.x; f < width; f += kBlock) {
-      float t = part[0][f];
-#pragma unroll
-      for (int w = 1; w < kWarpsPerBlock; ++w) t += part[w][f];
-      if (a.mean_rows) t *= rs;
-      if (SEG && a.accumulate) t += orow[f];
-      __stcs(orow + f, t);
-    }
-    __syncthreads();
+  heavy_rows<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+}
+
+// Blocks that walk the heavy list: as many as the device keeps resident, so that the heavy
+// segments (scheduled first, longest first) have the whole machine until the list runs out.
+template <typename K>
+int heavy_block_count(const Graph* g, K kernel, size_t smem) {
+  int per_sm = (int)g->heavy_blocks_per_sm;
+  if (per_sm <= 0) {
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kBlock, smem) != cudaSuccess)
+      per_sm = 2;
   }
-}
-
-// Kernel for graphs with short rows (the power-law workloads).  A warp still owns a run of
-// consecutive light rows, but the load steps ignore the row boundaries: every step fetches the
-// next U*NG edges of the run's contiguous edge stream, so a 3-edge row costs 3 loads, not a
-// predicated step of its own, and the loads of the next rows are already in flight while a row
-// is finished.  Row ends are found while the loaded vectors are added: a lane adds its vector
-// once its edge lies before the current row's end; when the row ends inside the step the lane
-// groups are combined, the row is stored and the accumulator restarts.  Few registers per
-// thread on purpose: with gathers that miss L2, resident warps are what keeps HBM busy.
-template <int VEC, int G, bool SCALED>
-__global__ void __launch_bounds__(kBlock) ap_flat_kernel(const ApArgs a) {
-  using V = typename Vec<VEC>::T;
-  constexpr int NG = 32 / G;
-  constexpr int U = NG >= 16 ? 2 : 4;
-  const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-  const int grp = lane / G;
-  const int c0 = lane % G;
-  const int f0 = blockIdx.y * a.slice_f;
-  const int chunks = (min(a.F, f0 + a.slice_f) - f0) / VEC;
-  const uint32_t row_bytes = (uint32_t)a.F * 4u;
-  const bool cok = c0 < chunks;  // lanes beyond the slice re-read vector 0 and never store
-  const char* xrow = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok ? c0 : 0) * VEC) * 4u;
-
-  const int rpw = a.rows_per_warp;
-  const int64_t rb = ((int64_t)blockIdx.x * kWarpsPerBlock + warp) * rpw;
-  if (rb >= a.n) return;
-  const int nrows = (int)min((int64_t)rpw, a.n - rb);
-  const int my_ptr = lane <= nrows ? (int)__ldg(a.ptr + rb + lane) : 0;
-  const int my_len = __shfl_down_sync(kFull, my_ptr, 1) - my_ptr;
-  const unsigned heavy_mask = __ballot_sync(kFull, lane < nrows && my_len > a.heavy_threshold);
-
-  V acc;
-  zero(acc);
-  auto store_row = [&](int i) {
-#pragma unroll
-    for (int off = G; off < 32; off <<= 1) add(acc, shfl_xor(acc, off));
-    const int len = __shfl_sync(kFull, my_len, i);
-    if (lane < G && cok) {
-      if (a.mean_rows) scale(acc, len > 0 ? 1.0f / (float)len : 1.0f);
-      stcs_vec(a.Y + (size_t)(rb + i) * (size_t)a.F + f0 + c0 * VEC, acc);
-    }
-    zero(acc);
-  };
-
-  int i0 = 0;
-  while (i0 < nrows) {
-    const unsigned later = heavy_mask >> i0;
-    const int i1 = later ? i0 + __ffs(later) - 1 : nrows;  // light rows [i0, i1)
-    if (i1 == i0) { ++i0; continue; }                       // a heavy block writes row i0
-    const int E0 = __shfl_sync(kFull, my_ptr, i0);
-    const int total = __shfl_sync(kFull, my_ptr, i1) - E0;
-    int32_t cur_u, nxt_u;
-    float cur_s, nxt_s;
-    load_batch<SCALED>(a, (int64_t)E0, E0 + total, lane, cur_u, cur_s);
-    load_batch<SCALED>(a, (int64_t)E0 + 32, E0 + total, lane, nxt_u, nxt_s);
-    int i = i0;
-    int hi_rel = __shfl_sync(kFull, my_ptr, i + 1) - E0;  // end of row i, in stream positions
-    for (int bpos = 0; bpos < total; bpos += 32) {
-      const int bcnt = min(32, total - bpos);
-      for (int s0 = 0; s0 < bcnt; s0 += U * NG) {
-        V v[U];
-        if (s0 + U * NG <= bcnt) {
-#pragma unroll
-          for (int j = 0; j < U; ++j) {
-            const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, s0 + j * NG + grp);
-            v[j] = ldg_vec(xrow + (uint64_t)u * row_bytes, V());
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < U; ++j) {
-            const int src = s0 + j * NG + grp;
-            const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src & 31);
-            if (src < bcnt) v[j] = ldg_vec(xrow + (uint64_t)u * row_bytes, V());
-            else zero(v[j]);
-          }
-        }
-#pragma unroll
-        for (int j = 0; j < U; ++j) {
-          const int pos0 = bpos + s0 + j * NG;  // first edge of this step; the same in all lanes
-          if (pos0 < total) {
-            const int lastpos = min(pos0 + NG, total) - 1;
-            const int mypos = pos0 + grp;
-            float sc = 1.f;
-            if (SCALED) sc = __shfl_sync(kFull, cur_s, (s0 + j * NG + grp) & 31);
-            bool todo = mypos <= lastpos;
-            for (;;) {
-              if (todo && mypos < hi_rel) {
-                if (SCALED) fma(acc, sc, v[j]);
-                else add(acc, v[j]);
-                todo = false;
-              }
-              if (hi_rel > lastpos) break;  // the current row goes on after this step
-              store_row(i);
-              ++i;
-              hi_rel = __shfl_sync(kFull, my_ptr, i + 1) - E0;
-            }
-          }
-        }
-      }
-      cur_u = nxt_u;
-      cur_s = nxt_s;
-      load_batch<SCALED>(a, (int64_t)E0 + bpos + 64, E0 + total, lane, nxt_u, nxt_s);
-    }
-    for (; i < i1; ++i) store_row(i);  // the row that ends with the stream, trailing empty rows
-    i0 = i1;
-  }
-}
-
-template <int VEC, int G, bool SCALED>
-dg_status_t launch_flat(const ApArgs& a, int slices, cudaStream_t s) {
-  const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
-  dim3 grid((unsigned)((a.n + rows_per_block - 1) / rows_per_block), (unsigned)slices);
-  ap_flat_kernel<VEC, G, SCALED><<<grid, kBlock, 0, s>>>(a);
-  DG_CUDA(cudaGetLastError());
-  count_launches(1);
-  return DG_OK;
-}
-
-template <int VEC, bool SCALED>
-dg_status_t dispatch_flat(const ApArgs& a, int slices, cudaStream_t s) {
-  const int chunks = (a.slice_f < a.F ? a.slice_f : a.F) / VEC;
-  if (chunks <= 2) return launch_flat<VEC, 2, SCALED>(a, slices, s);
-  if (chunks <= 4) return launch_flat<VEC, 4, SCALED>(a, slices, s);
-  if (chunks <= 8) return launch_flat<VEC, 8, SCALED>(a, slices, s);
-  if (chunks <= 16) return launch_flat<VEC, 16, SCALED>(a, slices, s);
-  return launch_flat<VEC, 32, SCALED>(a, slices, s);
+  return g->sm_count * (per_sm < 1 ? 1 : per_sm);
 }
 
 template <int VEC, int G, int CPL, bool SCALED>
 dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
   if (a.n == 0) return DG_OK;
-  const int heavy_blocks = g->sm_count * 2;
+  auto kernel = a.seg_lo ? ap_kernel<VEC, G, CPL, SCALED, true> : ap_kernel<VEC, G, CPL, SCALED, false>;
+  const int heavy_blocks = heavy_block_count(g, kernel, 0);
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
-  const int64_t blocks =
-      heavy_blocks + (a.heavy_only ? 0 : (a.n + rows_per_block - 1) / rows_per_block);
+  const int64_t blocks = heavy_blocks + (a.n + rows_per_block - 1) / rows_per_block;
   dim3 grid((unsigned)blocks, (unsigned)slices);
-  if (a.seg_lo) ap_kernel<VEC, G, CPL, SCALED, true><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
-  else ap_kernel<VEC, G, CPL, SCALED, false><<<grid, kBlock, 0, s>>>(a, heavy_blocks);
+  kernel<<<grid, kBlock, 0, s>>>(a, heavy_blocks);
   DG_CUDA(cudaGetLastError());
   count_launches(1);
   return DG_OK;
@@ -593,10 +510,6 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
       if (w >= 32) slice = w < slice ? w : slice;  // narrower than 128 bytes is not worth a pass
     }
   }
-  // Short rows and no source blocking: the flat-stream kernel, one vector per lane per slice.
-  const bool flat = nb == 1 && g->flat_rows != 0 &&
-                    (g->flat_rows == 1 || avg_len < (double)kFlatMaxAvgLen);
-  if (flat && slice > 32LL * vec) slice = 32LL * vec;
   slice = (slice / vec) * vec;
   if (slice < vec) slice = vec;
   // even out the slices: same count, smallest width that covers F
@@ -607,20 +520,6 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
   a.slice_f = (int32_t)slice;
   const int slices = (int)((a.F + slice - 1) / slice);
   const bool scaled = a.w != nullptr;
-
-  // Light rows by the flat-stream kernel; ap_kernel then keeps only the heavy list.
-  if (flat) {
-    ApArgs f = a;
-    int rpw = (int)g->flat_rows_per_warp;
-    if (rpw <= 0) rpw = (int)(256.0 / (avg_len > 1.0 ? avg_len : 1.0));  // ~256 edges per warp
-    f.rows_per_warp = rpw < 1 ? 1 : (rpw > 31 ? 31 : rpw);
-    dg_status_t st;
-    if (vec == 4) st = scaled ? dispatch_flat<4, true>(f, slices, s) : dispatch_flat<4, false>(f, slices, s);
-    else if (vec == 2) st = scaled ? dispatch_flat<2, true>(f, slices, s) : dispatch_flat<2, false>(f, slices, s);
-    else st = scaled ? dispatch_flat<1, true>(f, slices, s) : dispatch_flat<1, false>(f, slices, s);
-    if (st != DG_OK) return st;
-    a.heavy_only = 1;
-  }
 
   const int per = kFineBlocks / nb;
   for (int j = 0; j < nb; ++j) {

@@ -118,8 +118,8 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (g->heavy_cap > n) g->heavy_cap = n > 0 ? n : 1;
 
   e = cudaMalloc(&g->inv_deg, (size_t)(n > 0 ? n : 1) * sizeof(float));
-  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_rows, (size_t)g->heavy_cap * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)g->heavy_cap * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_rows, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->counters, 4 * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(g->counters, 0, 4 * sizeof(int32_t));
   if (e == cudaSuccess && wants_split(n, nnz))
@@ -312,14 +312,9 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     g->l2_budget_bytes = value << 20;
     return DG_OK;
   }
-  if (!strcmp(name, "flat_rows")) {
-    if (value < -1 || value > 1) return invalid("flat_rows must be -1 (automatic), 0 or 1");
-    g->flat_rows = value;
-    return DG_OK;
-  }
-  if (!strcmp(name, "flat_rows_per_warp")) {
-    if (value < 0 || value > 31) return invalid("flat_rows_per_warp must be in [0, 31]");
-    g->flat_rows_per_warp = value;
+  if (!strcmp(name, "heavy_blocks_per_sm")) {
+    if (value < 0 || value > 32) return invalid("heavy_blocks_per_sm must be in [0, 32]");
+    g->heavy_blocks_per_sm = value;
     return DG_OK;
   }
   if (!strcmp(name, "source_blocks")) {
@@ -338,8 +333,7 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
   if (!strcmp(name, "rows_per_block")) { *value = g->rows_per_block; return DG_OK; }
   if (!strcmp(name, "l2_budget_mb")) { *value = g->l2_budget_bytes >> 20; return DG_OK; }
   if (!strcmp(name, "source_blocks")) { *value = g->source_blocks; return DG_OK; }
-  if (!strcmp(name, "flat_rows")) { *value = g->flat_rows; return DG_OK; }
-  if (!strcmp(name, "flat_rows_per_warp")) { *value = g->flat_rows_per_warp; return DG_OK; }
+  if (!strcmp(name, "heavy_blocks_per_sm")) { *value = g->heavy_blocks_per_sm; return DG_OK; }
   return invalid("unknown parameter name");
 }
 

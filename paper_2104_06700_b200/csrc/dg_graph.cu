@@ -15,15 +15,48 @@ __global__ void inv_deg_kernel(const int64_t* __restrict__ rowptr, int64_t n,
   inv_deg[v] = d > 0 ? 1.0f / (float)d : 0.0f;
 }
 
-// Appends every segment longer than `threshold` to `list`.  The order of the list does not
-// influence any result: each heavy segment is summed by one block on its own.
-__global__ void heavy_list_kernel(const int64_t* __restrict__ ptr, int64_t n, int64_t threshold,
-                                  int32_t* __restrict__ list, int64_t cap,
-                                  int32_t* __restrict__ count) {
+// The heavy list holds every segment longer than `threshold`, longest first (in 64 length
+// classes, two per power of two): the blocks that walk it take entries x, x + B, x + 2B, ...,
+// so starting with the long ones evens out their finishing times.  The order of the list does
+// not influence any result: each heavy segment is summed by one block on its own.  The 64
+// class counters sit behind the list's `cap` entries.
+__device__ __forceinline__ int length_class(int64_t len) {
+  const int lg = 63 - __clzll(len);                     // len >= 1
+  const int half = lg > 0 ? (int)((len >> (lg - 1)) & 1) : 0;
+  const int c = 2 * lg + half;
+  return c > 63 ? 63 : c;
+}
+
+__global__ void heavy_count_kernel(const int64_t* __restrict__ ptr, int64_t n, int64_t threshold,
+                                   int32_t* __restrict__ classes, int32_t* __restrict__ count) {
   const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (v >= n) return;
-  if (ptr[v + 1] - ptr[v] > threshold) {
-    const int32_t slot = atomicAdd(count, 1);
+  const int64_t len = ptr[v + 1] - ptr[v];
+  if (len > threshold) {
+    atomicAdd(&classes[length_class(len)], 1);
+    atomicAdd(count, 1);
+  }
+}
+
+// One warp: classes[c] becomes the list position where class c starts (longest class first).
+__global__ void heavy_offsets_kernel(int32_t* __restrict__ classes) {
+  if (threadIdx.x != 0) return;
+  int32_t run = 0;
+  for (int c = 63; c >= 0; --c) {
+    const int32_t k = classes[c];
+    classes[c] = run;
+    run += k;
+  }
+}
+
+__global__ void heavy_fill_kernel(const int64_t* __restrict__ ptr, int64_t n, int64_t threshold,
+                                  int32_t* __restrict__ list, int64_t cap,
+                                  int32_t* __restrict__ classes) {
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= n) return;
+  const int64_t len = ptr[v + 1] - ptr[v];
+  if (len > threshold) {
+    const int32_t slot = atomicAdd(&classes[length_class(len)], 1);
     if (slot < cap) list[slot] = (int32_t)v;
   }
 }
@@ -98,11 +131,17 @@ dg_status_t build_degree_info(Graph* g, cudaStream_t s) {
 
 dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, int32_t* list,
                              int64_t cap, int32_t* count, cudaStream_t s) {
+  int32_t* classes = list + cap;  // 64 counters behind the list (see kHeavyListExtra)
   DG_CUDA(cudaMemsetAsync(count, 0, sizeof(int32_t), s));
+  DG_CUDA(cudaMemsetAsync(classes, 0, kHeavyListExtra * sizeof(int32_t), s));
   if (n == 0) return DG_OK;
-  heavy_list_kernel<<<blocks_for(n), kBlock, 0, s>>>(ptr, n, threshold, list, cap, count);
+  heavy_count_kernel<<<blocks_for(n), kBlock, 0, s>>>(ptr, n, threshold, classes, count);
   DG_CUDA(cudaGetLastError());
-  count_launches(1);
+  heavy_offsets_kernel<<<1, 32, 0, s>>>(classes);
+  DG_CUDA(cudaGetLastError());
+  heavy_fill_kernel<<<blocks_for(n), kBlock, 0, s>>>(ptr, n, threshold, list, cap, classes);
+  DG_CUDA(cudaGetLastError());
+  count_launches(3);
   return DG_OK;
 }
 

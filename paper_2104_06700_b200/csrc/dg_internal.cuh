@@ -20,7 +20,7 @@ struct dg_graph {
   int32_t* heavy_rows = nullptr; // CSR rows longer than heavy_threshold (forward)
   int32_t* heavy_cols = nullptr; // CSC columns longer than heavy_threshold (backward)
   int32_t* counters = nullptr;   // [0] #heavy rows, [1] #heavy cols, [2] validation flags
-  int64_t heavy_cap = 0;         // capacity of each heavy list
+  int64_t heavy_cap = 0;         // capacity of each heavy list (kHeavyListExtra more ints are allocated)
 
   // Source blocking: the neighbour ids are cut into kFineBlocks ranges of fine_rows ids;
   // split[b * n + v] is the first position of segment v whose neighbour id is >= b * fine_rows
@@ -44,19 +44,18 @@ struct dg_graph {
   int64_t heavy_built_for = 0;   // threshold the heavy lists were built with
   int64_t slice_features = 0;    // 0 = automatic
   int64_t rows_per_block = 32;
+  int64_t heavy_blocks_per_sm = 0;  // blocks per SM that walk the heavy list; 0 = all resident ones
   int64_t l2_budget_bytes = 0;   // bytes of the gathered matrix one launch may keep L2-resident
   int64_t source_blocks = 0;     // 0 = automatic, else 1, 2, 4, 8 or 16
-  int64_t flat_rows = -1;        // flat-stream kernel for short rows: -1 = automatic, 0 = off, 1 = on
-  int64_t flat_rows_per_warp = 0;  // 0 = about 256 edges per warp
 };
 
 namespace dg {
 
 using Graph = ::dg_graph;
 
+constexpr int kHeavyListExtra = 64;      // counters of the length classes, stored behind a heavy list
 constexpr int kFineBlocks = 16;          // finest cut of the neighbour ids for source blocking
 constexpr int64_t kBlockingMinAvgLen = 64;  // split pointers are built when nnz >= 64 n
-constexpr int64_t kFlatMaxAvgLen = 128;     // below this average row length: flat-stream kernel
 
 // One direction of AP as the kernels see it: out[r] = rs_r * sum_k s_k * X[idx[k]],
 // s_k = w[k] (1 when w is absent).
@@ -78,7 +77,6 @@ struct ApArgs {
   const int32_t* seg_lo;      // source-blocked pass: first and one-past-last position of every
   const int32_t* seg_hi;      //   segment's piece (n entries each); nullptr = whole segments
   int32_t accumulate;         // source-blocked pass after the first: add to what Y holds
-  int32_t heavy_only;         // launch only the blocks that walk the heavy list
 };
 
 void set_error(const std::string& msg);

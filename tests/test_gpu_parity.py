@@ -49,14 +49,9 @@ def test_tiny_transpose_bit_exact(tiny, weighted):
 @pytest.mark.parametrize("F", [64, 8, 100, 602, 256, 128, 1, 3, 6, 130, 1028])
 @pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
 @pytest.mark.parametrize("weighted", [True, False])
-@pytest.mark.parametrize("flat", [0, 1])
-def test_tiny_forward_backward(tiny, F, op, weighted, flat):
-    """flat = 1: the kernel whose load steps run over row boundaries (what short rows get by
-    default); flat = 0: the row-by-row kernel."""
+def test_tiny_forward_backward(tiny, F, op, weighted):
     sg = tiny if weighted else synth.make("tiny", weighted=False)
     g = make_graph(sg)
-    g.dg_graph_set_param("flat_rows", flat)
-    g.dg_graph_set_param("heavy_threshold", 256)
     csc = check_transpose(g, *host_csr(sg))
     H = synth.features(sg.n, F, 100 + F, DEV)
     G = synth.features(sg.n, F, 200 + F, DEV)
@@ -74,24 +69,23 @@ def test_tiny_deterministic_bits(tiny):
     assert torch.equal(a, b) and torch.equal(c, d)
 
 
-@pytest.mark.parametrize("slice_f,heavy,rows_per_block", [(16, 64, 1), (32, 64, 8), (0, 128, 64),
-                                                         (600, 1024, 32), (4, 4096, 3)])
-def test_tiny_launch_shapes(tiny, slice_f, heavy, rows_per_block):
+@pytest.mark.parametrize("slice_f,heavy,rows_per_block,heavy_blocks",
+                         [(16, 64, 1, 0), (32, 64, 8, 1), (0, 128, 64, 3), (600, 1024, 32, 0),
+                          (4, 4096, 3, 2)])
+def test_tiny_launch_shapes(tiny, slice_f, heavy, rows_per_block, heavy_blocks):
     """Feature slicing, the heavy-segment path and the block shape change the launch, not the
     result (columns of the tiny graph reach 488 entries, above the lowered heavy threshold)."""
     g = make_graph(tiny)
     g.dg_graph_set_param("heavy_threshold", heavy)
     g.dg_graph_set_param("slice_features", slice_f)
     g.dg_graph_set_param("rows_per_block", rows_per_block)
+    g.dg_graph_set_param("heavy_blocks_per_sm", heavy_blocks)
     assert g.dg_graph_get_param("heavy_threshold") == heavy
     csc = check_transpose(g, *host_csr(tiny))
-    for flat, rpw in ((0, 0), (1, 0), (1, 1), (1, 31)):
-        g.dg_graph_set_param("flat_rows", flat)
-        g.dg_graph_set_param("flat_rows_per_warp", rpw)
-        for F in (64, 602, 10):
-            H = synth.features(tiny.n, F, 5, DEV)
-            G = synth.features(tiny.n, F, 6, DEV)
-            check_fwd_bwd(g, host_csr(tiny), H, G, binding.DG_OP_MEAN, csc)
+    for F in (64, 602, 10):
+        H = synth.features(tiny.n, F, 5, DEV)
+        G = synth.features(tiny.n, F, 6, DEV)
+        check_fwd_bwd(g, host_csr(tiny), H, G, binding.DG_OP_MEAN, csc)
 
 
 def test_unaligned_feature_pointers(tiny):
@@ -127,15 +121,13 @@ def test_identity_and_ring_bit_exact():
 
 
 @pytest.mark.parametrize("F", [8, 100, 602])
-@pytest.mark.parametrize("flat", [0, 1])
-def test_star_graph_heavy_row_and_column(F, flat):
+def test_star_graph_heavy_row_and_column(F):
     """Vertex 0 pulls from every other vertex (one CSR row of n-1 entries, a heavy row), and
     every other vertex pulls from vertex 1 (one CSC column of n-1 entries)."""
     n = 6000
     rows = [list(range(1, n))] + [[1] for _ in range(n - 1)]
     w = np.random.default_rng(0).random(2 * (n - 1)).astype(np.float32)
     g, rowptr, colidx = csr_graph(n, rows, weights=w)
-    g.dg_graph_set_param("flat_rows", flat)
     csc = check_transpose(g, rowptr, colidx, w)
     H = synth.features(n, F, 11, DEV)
     G = synth.features(n, F, 12, DEV)
@@ -186,24 +178,6 @@ def test_unsorted_rows_duplicates_and_self_loops():
     csc = check_transpose(g, rowptr, src, w)
     H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
     check_fwd_bwd(g, (rowptr, src, w), H, G, binding.DG_OP_MEAN, csc)
-
-
-# ------------------------------------------------------------------ flat-stream kernel
-def test_flat_kernel_empty_rows_and_deterministic_bits():
-    """Rows of 0..39 edges, every third row empty: runs of empty rows inside and at the end of a
-    warp's stream; the same call twice gives the same bits."""
-    n, F = 3000, 64
-    rng = np.random.default_rng(3)
-    rows = [sorted(rng.choice(n, rng.integers(0, 40), replace=False).tolist()) if v % 3 else []
-            for v in range(n)]
-    g, rowptr, colidx = csr_graph(n, rows)
-    g.dg_graph_set_param("flat_rows", 1)
-    csc = check_transpose(g, rowptr, colidx, None)
-    for F in (64, 20, 200):
-        H, G = synth.features(n, F, 1, DEV), synth.features(n, F, 2, DEV)
-        check_fwd_bwd(g, (rowptr, colidx, None), H, G, binding.DG_OP_MEAN, csc)
-    a = g.dg_aggregate_fwd(H, binding.DG_OP_SUM).clone()
-    assert torch.equal(a, g.dg_aggregate_fwd(H, binding.DG_OP_SUM))
 
 
 # ------------------------------------------------------------------ source blocking
