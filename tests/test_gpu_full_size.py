@@ -1,0 +1,209 @@
+"""GPU parity at the full sizes of the benchmark workloads, in the launch configuration bench.py
+times (default knobs).
+
+Configs 2-4 (Reddit-, Products- and Proteins-like): the CSC is compared with the oracle's stable
+counting sort in full, bit for bit; forward and backward AP are compared with the oracle on a
+sample of output rows (random rows plus the longest ones, which take the block-per-row path).
+Every output row depends only on its own CSR row (CSC column), so the oracle can compute the
+sampled rows one by one: it is given the sub-problem made of those rows, with the neighbour ids
+renumbered into the compact matrix of the rows they reference.
+
+Config 5 (Papers-like, 1.6 G edges): the host cannot hold the oracle's inputs, so the CSC is
+checked through the properties that define it uniquely (perm is a permutation; keys
+non-decreasing along perm; perm increasing inside equal keys; colptr = key boundaries;
+rowidx_T = row of perm), evaluated with torch on the GPU, and AP on sampled rows as above.
+
+Set DG_SKIP_FULL_SIZE=1 to skip these (they take a few minutes).
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2104_06700_b200 import binding, synth
+from parity_util import assert_within_bound, to_np
+
+pytestmark = [pytest.mark.gpu,
+              pytest.mark.skipif(os.environ.get("DG_SKIP_FULL_SIZE") == "1",
+                                 reason="DG_SKIP_FULL_SIZE=1")]
+DEV = "cuda"
+
+
+def sample_segments(ptr, idx, w, seg_ids):
+    """Sub-problem of the segments `seg_ids` of a CSR/CSC given as torch tensors on the GPU.
+    Returns host arrays (sub_ptr, sub_idx renumbered, sub_w) and the GPU tensor of the distinct
+    neighbour ids, in the order of the renumbering."""
+    seg = torch.as_tensor(seg_ids, device=ptr.device, dtype=torch.int64)
+    lo, hi = ptr[seg], ptr[seg + 1]
+    lens = hi - lo
+    sub_ptr = torch.zeros(seg.numel() + 1, dtype=torch.int64, device=ptr.device)
+    torch.cumsum(lens, 0, out=sub_ptr[1:])
+    total = int(sub_ptr[-1])
+    # positions of all edges of the sampled segments, segment by segment, in order
+    owner = torch.repeat_interleave(torch.arange(seg.numel(), device=ptr.device), lens)
+    pos = lo[owner] + (torch.arange(total, device=ptr.device) - sub_ptr[owner])
+    nb = idx[pos].long()
+    uniq, inv = torch.unique(nb, return_inverse=True)
+    sub_w = None if w is None else to_np(w[pos])
+    return to_np(sub_ptr), to_np(inv.to(torch.int32)), sub_w, uniq, pos
+
+
+def pick_rows(ptr, n, count, longest, seed):
+    lens = ptr[1:] - ptr[:-1]
+    top = torch.topk(lens, min(longest, n)).indices
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    rnd = torch.randperm(n, generator=gen)[:count].to(ptr.device)
+    return torch.unique(torch.cat([top, rnd])).cpu().numpy()
+
+
+def _pad_ptr(ptr, n_sub):
+    """Row pointer of a sub-problem extended by empty segments up to n_sub segments."""
+    out = np.full(n_sub + 1, ptr[-1], dtype=np.int64)
+    out[:len(ptr)] = ptr
+    return out
+
+
+def _pad_rows(M, n_sub):
+    out = np.zeros((n_sub, M.shape[1]), dtype=np.float32)
+    out[:M.shape[0]] = M
+    return out
+
+
+def check_sampled(g, sg, H, G, op, rows, cols):
+    """Forward on sampled destination rows, backward on sampled source columns.  The oracle
+    gets a sub-problem whose vertices 0..k-1 are the sampled segments (the others are empty) and
+    whose neighbour ids are renumbered into the compact matrix of referenced rows."""
+    colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
+    out = g.dg_aggregate_fwd(H, op)
+    sp, si, sw, uniq, _ = sample_segments(sg.rowptr, sg.colidx, sg.edge_w, rows)
+    n_sub = max(len(rows), uniq.numel())
+    ref, mag = oracle.ap_forward(_pad_ptr(sp, n_sub), si, sw, _pad_rows(to_np(H[uniq]), n_sub), op,
+                                 rows=np.arange(len(rows)))
+    worst_f = assert_within_bound(to_np(out[torch.as_tensor(rows, device=DEV)]), ref, mag, "fwd")
+    del out
+    dH = g.dg_aggregate_bwd(G, op)
+    sp, si, sw, uniq, _ = sample_segments(colptr, rowidx_T, w_T, cols)
+    n_sub = max(len(cols), uniq.numel())
+    # the mean's divisor belongs to the destination vertex: the oracle reads it from a CSR row
+    # pointer, here one that gives every renumbered destination its true in-degree
+    deg = to_np(sg.rowptr[uniq + 1] - sg.rowptr[uniq])
+    rp = np.zeros(n_sub + 1, dtype=np.int64)
+    rp[1:len(deg) + 1] = np.cumsum(deg)
+    rp[len(deg) + 1:] = rp[len(deg)]
+    ref, mag = oracle.ap_backward(rp, _pad_ptr(sp, n_sub), si, sw,
+                                  _pad_rows(to_np(G[uniq]), n_sub), op, cols=np.arange(len(cols)))
+    worst_b = assert_within_bound(to_np(dH[torch.as_tensor(cols, device=DEV)]), ref, mag, "bwd")
+    return worst_f, worst_b
+
+
+@pytest.mark.parametrize("name,F,ops", [
+    ("reddit_like", 602, (binding.DG_OP_MEAN,)),
+    ("products_like", 100, (binding.DG_OP_SUM, binding.DG_OP_MEAN)),
+    ("proteins_like", 64, (binding.DG_OP_SUM,)),
+])
+def test_full_size_csc_bit_exact_and_sampled_rows(name, F, ops):
+    sg = synth.make(name, device=DEV)
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+    g.dg_graph_validate()
+    g.dg_graph_transpose()
+    torch.cuda.synchronize()
+    colptr, rowidx_T, w_T, perm = g.dg_graph_get_csc()
+    o_colptr, o_rowidx, o_w, o_perm = oracle.transpose(
+        to_np(sg.rowptr), to_np(sg.colidx), to_np(sg.edge_w))
+    assert np.array_equal(to_np(colptr), o_colptr), "colptr"
+    assert np.array_equal(to_np(rowidx_T), o_rowidx), "rowidx_T"
+    assert np.array_equal(to_np(perm).astype(np.int64), o_perm), "perm"
+    if sg.edge_w is not None:
+        assert to_np(w_T).tobytes() == o_w.tobytes(), "w_T"
+    del o_colptr, o_rowidx, o_w, o_perm
+    H = synth.features(sg.n, F, 61, DEV)
+    G = synth.features(sg.n, F, 62, DEV)
+    rows = pick_rows(sg.rowptr, sg.n, 1500, 40, 7)
+    cols = pick_rows(colptr, sg.n, 1500, 40, 8)
+    for op in ops:
+        wf, wb = check_sampled(g, sg, H, G, op, rows, cols)
+        assert wf <= 1.0 and wb <= 1.0
+    # the library's widths for the other layers of the same graph
+    if name == "proteins_like":
+        for F2 in (8, 256):
+            H2, G2 = synth.features(sg.n, F2, 63, DEV), synth.features(sg.n, F2, 64, DEV)
+            check_sampled(g, sg, H2, G2, binding.DG_OP_SUM, rows[:400], cols[:400])
+
+
+def _check_csc_properties(sg, colptr, rowidx_T, perm, chunk=1 << 27):
+    """The five properties that pin the CSC uniquely, evaluated with torch on the GPU in chunks.
+    perm is int32 on the device (edge positions fit 31 bits)."""
+    n, nnz = sg.n, sg.nnz
+    seen = torch.zeros(nnz, dtype=torch.bool, device=DEV)
+    prev_key = torch.full((1,), -1, dtype=torch.int64, device=DEV)
+    prev_pos = torch.full((1,), -1, dtype=torch.int64, device=DEV)
+    counts = torch.zeros(n, dtype=torch.int64, device=DEV)
+    for s in range(0, nnz, chunk):
+        e = min(nnz, s + chunk)
+        p = perm[s:e].long()
+        assert int(p.min()) >= 0 and int(p.max()) < nnz
+        seen[p] = True
+        key = sg.colidx[p].long()
+        k_ext = torch.cat([prev_key, key])
+        p_ext = torch.cat([prev_pos, p])
+        dk = k_ext[1:] - k_ext[:-1]
+        assert bool((dk >= 0).all()), "keys decrease along perm"
+        same = dk == 0
+        assert bool(((p_ext[1:] - p_ext[:-1])[same] > 0).all()), "unstable order inside a column"
+        # rowidx_T[q] is the row r with rowptr[r] <= perm[q] < rowptr[r+1]
+        r = torch.searchsorted(sg.rowptr, p, right=True) - 1
+        assert torch.equal(r.to(torch.int32), rowidx_T[s:e]), "rowidx_T"
+        counts += torch.bincount(key, minlength=n)
+        prev_key, prev_pos = key[-1:].clone(), p[-1:].clone()
+        del p, key, k_ext, p_ext, dk, same, r
+    assert bool(seen.all()), "perm is not a permutation"
+    del seen
+    expect = torch.zeros(n + 1, dtype=torch.int64, device=DEV)
+    torch.cumsum(counts, 0, out=expect[1:])
+    assert torch.equal(expect, colptr), "colptr"
+
+
+def test_papers_like_full_size():
+    """111 M vertices, 1.6 G edges, F = 128, sum: CSC by its defining properties, AP on sampled
+    rows and columns; two feature buffers as in the benchmark (backward reads the forward's
+    input and overwrites its output)."""
+    free, total = torch.cuda.mem_get_info()
+    if total < 170e9:
+        pytest.skip("needs a 180 GB device")
+    sg = synth.make("papers_like", device=DEV)
+    torch.cuda.empty_cache()
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, None)
+    g.dg_graph_validate()
+    need_csc, need_scratch = g.dg_graph_transpose_workspace()
+    csc = torch.empty(need_csc, dtype=torch.uint8, device=DEV)
+    scratch = torch.empty(need_scratch, dtype=torch.uint8, device=DEV)
+    g.dg_graph_transpose(csc, scratch)
+    torch.cuda.synchronize()
+    del scratch
+    torch.cuda.empty_cache()
+    colptr, rowidx_T, w_T, perm = g.dg_graph_get_csc()
+    assert w_T is None
+    _check_csc_properties(sg, colptr, rowidx_T, perm)
+    torch.cuda.empty_cache()
+    F = 128
+    H = synth.features(sg.n, F, 71, DEV)
+    out = torch.empty_like(H)
+    rows = pick_rows(sg.rowptr, sg.n, 3000, 30, 9)
+    cols = pick_rows(colptr, sg.n, 3000, 30, 10)
+    g.dg_aggregate_fwd(H, binding.DG_OP_SUM, out=out)
+    sp, si, _, uniq, _ = sample_segments(sg.rowptr, sg.colidx, None, rows)
+    n_sub = max(len(rows), uniq.numel())
+    ref, mag = oracle.ap_forward(_pad_ptr(sp, n_sub), si, None, _pad_rows(to_np(H[uniq]), n_sub),
+                                 oracle.OP_SUM, rows=np.arange(len(rows)))
+    assert_within_bound(to_np(out[torch.as_tensor(rows, device=DEV)]), ref, mag, "fwd")
+    g.dg_aggregate_bwd(H, binding.DG_OP_SUM, dH=out)
+    sp, si, _, uniq, _ = sample_segments(colptr, rowidx_T, None, cols)
+    n_sub = max(len(cols), uniq.numel())
+    rp = np.zeros(n_sub + 1, dtype=np.int64)          # sum: the divisor is not used
+    ref, mag = oracle.ap_backward(rp, _pad_ptr(sp, n_sub), si, None,
+                                  _pad_rows(to_np(H[uniq]), n_sub), oracle.OP_SUM,
+                                  cols=np.arange(len(cols)))
+    assert_within_bound(to_np(out[torch.as_tensor(cols, device=DEV)]), ref, mag, "bwd")
