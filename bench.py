@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--feat", type=int, default=0, help="feature width (0 = the workload's)")
     ap.add_argument("--op", default=None, choices=[None, "sum", "mean"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--epochs", type=int, default=5,
+                    help="GraphSAGE epochs to time after 3 warm-up epochs (0 = skip)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0,
                     help="target CPU time of the oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -318,6 +320,36 @@ def main():
         "gather_GBs": sg.nnz * F * 4 / (dom_ms * 1e-3) / 1e9,
     }
 
+    # ---------------------------------------------------------------- GraphSAGE epoch (composite)
+    epoch_info = None
+    epoch_dims = {"reddit_like": [602, 256, 41], "products_like": [100, 256, 256, 47]}
+    if args.epochs > 0 and args.workload in epoch_dims and not args.feat and not two_buffers:
+        from paper_2104_06700_b200 import graphsage
+        dims = epoch_dims[args.workload]
+        frac = 0.65 if args.workload == "reddit_like" else 196615 / 2449029
+        torch.manual_seed(1234)
+        model = graphsage.GraphSAGE(g, dims).to(dev)
+        labels = torch.randint(0, dims[-1], (sg.n,), device=dev)
+        train_idx = torch.nonzero(torch.rand(sg.n, device=dev) < frac).flatten()
+        run_epoch = graphsage.make_epoch(model, H, labels, train_idx)
+        for _ in range(3):
+            run_epoch()
+        torch.cuda.synchronize()
+        a, b = ev(), ev()
+        a.record(stream)
+        for _ in range(args.epochs):
+            last_loss = run_epoch()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ep_ms = a.elapsed_time(b) / args.epochs
+        calls = graphsage.aggregation_calls(dims)
+        epoch_info = {"ms_per_epoch": ep_ms, "epochs": args.epochs, "dims": dims,
+                      "train_vertices": int(train_idx.numel()), "loss": float(last_loss),
+                      "aggregations": [f"{d}:{w}" for d, w in calls],
+                      "ap_edge_feat_per_epoch": sg.nnz * sum(w for _, w in calls),
+                      "aggregator": "(sum + self) / (deg + 1), then Linear; ReLU; Adam"}
+        del model, run_epoch
+
     # ---------------------------------------------------------------- end to end from host memory
     e2e = None
     if two_buffers:
@@ -383,7 +415,7 @@ def main():
                        if sg.n * F * 4 > 252e6 else "inputs fit L2: warm-L2 numbers",
                        "knobs": args.set},
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-            "clocks": clocks,
+            "clocks": clocks, "epoch": epoch_info,
             "ingest": {"graph_create_ms": create_ms, "transpose_ms": transpose_ms,
                        "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3) if transpose_ms else None},
         }))
