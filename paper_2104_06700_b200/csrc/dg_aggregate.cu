@@ -257,9 +257,9 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_bloc
 // rows_per_warp consecutive light segments and streams their indices as one run of 32-edge
 // batches, the next batch always in flight while the current one is summed.
 template <int VEC, int G, int CPL, bool SCALED, bool SEG>
-__global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
+__device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
+                                        float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
   using V = typename Vec<VEC>::T;
-  __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int grp = lane / G;
@@ -410,6 +410,23 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
   heavy_rows<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
 
+template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+__global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
+  __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
+  ap_body<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+}
+
+// The same kernel compiled for five resident blocks per SM (at most 48 registers).  The scaled
+// variants with up to four floats per lane and step (and at least 16 lanes per edge) carry the edge factors on top of everything
+// else and would take 60 registers; measured on B200 the higher occupancy wins for them
+// (Reddit-like backward 22.0 -> 19.3 ms, Products-like backward 7.0 -> 6.2 ms), while the same
+// cap slows the unscaled variants down.
+template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+__global__ void __launch_bounds__(kBlock, 5) ap_kernel_r48(const ApArgs a, const int heavy_blocks) {
+  __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
+  ap_body<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+}
+
 // Blocks that walk the heavy list: as many as the device keeps resident, so that the heavy
 // segments (scheduled first, longest first) have the whole machine until the list runs out.
 template <typename K>
@@ -425,7 +442,13 @@ int heavy_block_count(const Graph* g, K kernel, size_t smem) {
 template <int VEC, int G, int CPL, bool SCALED>
 dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
   if (a.n == 0) return DG_OK;
-  auto kernel = a.seg_lo ? ap_kernel<VEC, G, CPL, SCALED, true> : ap_kernel<VEC, G, CPL, SCALED, false>;
+  void (*kernel)(const ApArgs, const int);
+  if constexpr (SCALED && VEC * CPL <= 4 && G >= 16) {
+    kernel = a.seg_lo ? ap_kernel_r48<VEC, G, CPL, SCALED, true>
+                      : ap_kernel_r48<VEC, G, CPL, SCALED, false>;
+  } else {
+    kernel = a.seg_lo ? ap_kernel<VEC, G, CPL, SCALED, true> : ap_kernel<VEC, G, CPL, SCALED, false>;
+  }
   const int heavy_blocks = heavy_block_count(g, kernel, 0);
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
   const int64_t blocks = heavy_blocks + (a.n + rows_per_block - 1) / rows_per_block;
