@@ -153,13 +153,17 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
 
 /*
  * Forward and backward AP with the feature matrices in HOST memory (pinned memory makes the
- * copies asynchronous and faster; pageable memory works).  Equivalent to copying H_host and
- * dOut_host into device_ws, calling dg_aggregate_fwd and dg_aggregate_bwd, and copying the
- * results into out_host and dH_host, all on `stream`.  dOut_host/dH_host may both be NULL to
- * run the forward pass only.
- *   device_ws  device, 256-byte aligned, >= dg_aggregate_host_workspace(g, F) bytes
- * Asynchronous on `stream` when the host buffers are pinned; the host results are complete
- * once the stream has been synchronised.
+ * copies asynchronous and lets them overlap the kernels; pageable memory works but serialises).
+ * Computes what dg_aggregate_fwd on H_host and dg_aggregate_bwd on dOut_host compute and leaves
+ * the results in out_host and dH_host.  The feature columns are independent in AP, so matrices
+ * wider than 256 columns travel in chunks of 128 columns: a chunk is uploaded while the previous
+ * one is aggregated and the one before that is downloaded, on two helper streams the handle
+ * creates at its first call of this function.  (The summation order inside an output element
+ * can therefore differ from a full-width call; both are within the stated error bound.)
+ * Everything is ordered after the work already queued on `stream`, and `stream` finishing means
+ * all copies are done.  dOut_host/dH_host may both be NULL to run the forward pass only.
+ *   device_ws  device, 256-byte aligned, >= dg_aggregate_host_workspace(g, F) bytes (four
+ *              n x F matrices at most)
  */
 size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F);
 dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dOut_host,

@@ -37,6 +37,12 @@ static dg_status_t free_owned(Graph* g) {
   if (g->counters) cudaFree(g->counters);
   if (g->split_csr) cudaFree(g->split_csr);
   g->split_csr = nullptr;
+  for (cudaEvent_t e : g->aux_events) cudaEventDestroy(e);
+  g->aux_events.clear();
+  if (g->aux_ready) {
+    for (int i = 0; i < 2; ++i) cudaStreamDestroy(g->aux_stream[i]);
+    g->aux_ready = false;
+  }
   g->inv_deg = nullptr;
   g->heavy_rows = g->heavy_cols = g->counters = nullptr;
   return DG_OK;
@@ -256,9 +262,29 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
 size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F) {
   if (!g || F < 1) return 0;
   const size_t mat = (((size_t)g->n * (size_t)F * sizeof(float)) + 255) & ~(size_t)255;
-  return 2 * (mat > 0 ? mat : 256);
+  return 4 * (mat > 0 ? mat : 256);
 }
 
+// Helper streams (upload, download) and a pool of events per handle, created on first use.
+static dg_status_t host_pipeline(Graph* g, size_t events) {
+  if (!g->aux_ready) {
+    for (int i = 0; i < 2; ++i)
+      DG_CUDA(cudaStreamCreateWithFlags(&g->aux_stream[i], cudaStreamNonBlocking));
+    g->aux_ready = true;
+  }
+  while (g->aux_events.size() < events) {
+    cudaEvent_t e;
+    DG_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    g->aux_events.push_back(e);
+  }
+  return DG_OK;
+}
+
+// The feature columns are independent of each other in AP, so the host matrices travel in column
+// chunks: chunk c of H is uploaded (a strided copy into a compact n x w matrix) while chunk c-1 is
+// being aggregated and the result of chunk c-2 is on its way back; then the same for dOut.  PCIe
+// carries both directions at once, so a call costs about max(kernel time, copy time) instead of
+// their sum.  Two input and two output chunk buffers alternate.
 dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dOut_host,
                               int32_t F, dg_op_t op, float* out_host, float* dH_host,
                               void* device_ws, size_t device_ws_bytes, void* stream) {
@@ -272,19 +298,63 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
     set_error("device_ws smaller than dg_aggregate_host_workspace reports");
     return DG_ERR_WORKSPACE;
   }
-  cudaStream_t s = (cudaStream_t)stream;
-  const size_t bytes = (size_t)g->n * (size_t)F * sizeof(float);
-  const size_t mat = dg_aggregate_host_workspace(g, F) / 2;
-  float* d_in = reinterpret_cast<float*>(device_ws);
-  float* d_out = reinterpret_cast<float*>(static_cast<char*>(device_ws) + mat);
-  if (bytes) DG_CUDA(cudaMemcpyAsync(d_in, H_host, bytes, cudaMemcpyHostToDevice, s));
-  if (dg_status_t st = dg_aggregate_fwd(g, d_in, F, op, d_out, stream)) return st;
-  if (bytes) DG_CUDA(cudaMemcpyAsync(out_host, d_out, bytes, cudaMemcpyDeviceToHost, s));
-  if (dOut_host) {
-    if (bytes) DG_CUDA(cudaMemcpyAsync(d_in, dOut_host, bytes, cudaMemcpyHostToDevice, s));
-    if (dg_status_t st = dg_aggregate_bwd(g, d_in, F, op, d_out, stream)) return st;
-    if (bytes) DG_CUDA(cudaMemcpyAsync(dH_host, d_out, bytes, cudaMemcpyDeviceToHost, s));
+  if (dOut_host && !g->transposed) {
+    set_error("the backward pass needs dg_graph_transpose first");
+    return DG_ERR_NOT_TRANSPOSED;
   }
+  if (g->n == 0) return DG_OK;
+  // chunk width: 128 columns (one 512-byte row slice) once the matrix is wider than 256 columns
+  const int32_t W = F > 256 ? 128 : F;
+  const int chunks = (F + W - 1) / W;
+  const int tasks = chunks * (dOut_host ? 2 : 1);
+  if (dg_status_t st = host_pipeline(g, 1 + 3 * (size_t)tasks)) return st;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaStream_t up = g->aux_stream[0], down = g->aux_stream[1];
+  cudaEvent_t* ev = g->aux_events.data();
+  cudaEvent_t start = ev[0];
+  auto uploaded = [&](int t) { return ev[1 + 3 * t]; };
+  auto computed = [&](int t) { return ev[2 + 3 * t]; };
+  auto downloaded = [&](int t) { return ev[3 + 3 * t]; };
+
+  const size_t buf = (((size_t)g->n * (size_t)W * sizeof(float)) + 255) & ~(size_t)255;
+  char* ws = static_cast<char*>(device_ws);
+  float* d_in[2] = {reinterpret_cast<float*>(ws), reinterpret_cast<float*>(ws + buf)};
+  float* d_out[2] = {reinterpret_cast<float*>(ws + 2 * buf), reinterpret_cast<float*>(ws + 3 * buf)};
+  const size_t host_pitch = (size_t)F * sizeof(float);
+
+  // everything queued on `stream` so far (an earlier call may still use the workspace) comes first
+  DG_CUDA(cudaEventRecord(start, s));
+  DG_CUDA(cudaStreamWaitEvent(up, start, 0));
+  DG_CUDA(cudaStreamWaitEvent(down, start, 0));
+  for (int t = 0; t < tasks; ++t) {
+    const bool bwd = t >= chunks;
+    const int c = bwd ? t - chunks : t;
+    const int32_t w = (c + 1) * W <= F ? W : F - c * W;
+    const float* src = (bwd ? dOut_host : H_host) + (size_t)c * W;
+    float* dst = (bwd ? dH_host : out_host) + (size_t)c * W;
+    float* in = d_in[t & 1];
+    float* out = d_out[t & 1];
+    // upload: the input buffer is free once the kernels of task t-2 have read it
+    if (t >= 2) DG_CUDA(cudaStreamWaitEvent(up, computed(t - 2), 0));
+    DG_CUDA(cudaMemcpy2DAsync(in, (size_t)w * sizeof(float), src, host_pitch,
+                              (size_t)w * sizeof(float), (size_t)g->n, cudaMemcpyHostToDevice, up));
+    DG_CUDA(cudaEventRecord(uploaded(t), up));
+    // compute: needs the upload, and the output buffer back from the download of task t-2
+    DG_CUDA(cudaStreamWaitEvent(s, uploaded(t), 0));
+    if (t >= 2) DG_CUDA(cudaStreamWaitEvent(s, downloaded(t - 2), 0));
+    if (dg_status_t st = bwd ? dg_aggregate_bwd(g, in, w, op, out, stream)
+                             : dg_aggregate_fwd(g, in, w, op, out, stream))
+      return st;
+    DG_CUDA(cudaEventRecord(computed(t), s));
+    // download
+    DG_CUDA(cudaStreamWaitEvent(down, computed(t), 0));
+    DG_CUDA(cudaMemcpy2DAsync(dst, host_pitch, out, (size_t)w * sizeof(float),
+                              (size_t)w * sizeof(float), (size_t)g->n, cudaMemcpyDeviceToHost, down));
+    DG_CUDA(cudaEventRecord(downloaded(t), down));
+  }
+  // `stream` finishing means every copy has finished
+  DG_CUDA(cudaStreamWaitEvent(s, downloaded(tasks - 1), 0));
+  if (tasks >= 2) DG_CUDA(cudaStreamWaitEvent(s, downloaded(tasks - 2), 0));
   return DG_OK;
 }
 

@@ -6,6 +6,7 @@
 
 #include <atomic>
 #include <string>
+#include <vector>
 
 #include "dg.h"
 
@@ -29,6 +30,11 @@ struct dg_graph {
   int32_t* split_csr = nullptr;
   int32_t* split_csc = nullptr;
   int64_t fine_rows = 0;
+
+  // dg_aggregate_host: helper streams (upload, download) and events, created on first use
+  bool aux_ready = false;
+  cudaStream_t aux_stream[2] = {nullptr, nullptr};
+  std::vector<cudaEvent_t> aux_events;
 
   bool transposed = false;
   const int64_t* colptr = nullptr;

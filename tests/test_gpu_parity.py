@@ -280,6 +280,38 @@ def test_host_entry_point(tiny):
     assert torch.equal(dH, g.dg_aggregate_bwd(G.to(DEV), binding.DG_OP_MEAN).cpu())
 
 
+@pytest.mark.parametrize("F,pinned", [(602, True), (300, True), (257, False)])
+def test_host_entry_point_in_column_chunks(tiny, F, pinned):
+    """Matrices wider than 256 columns go through the host entry point in 128-column chunks
+    (upload, kernels and download overlapped); the result is checked against the oracle, twice in
+    a row so that the second call reuses the workspace while the first may still be draining."""
+    g = make_graph(tiny)
+    csc = check_transpose(g, *host_csr(tiny))
+    H = synth.features(tiny.n, F, 1)
+    G = synth.features(tiny.n, F, 2)
+    if pinned:
+        H, G = H.pin_memory(), G.pin_memory()
+    out, dH = torch.empty_like(H), torch.empty_like(H)
+    if pinned:
+        out, dH = out.pin_memory(), dH.pin_memory()
+    ws = torch.empty(g.dg_aggregate_host_workspace(F), dtype=torch.uint8, device=DEV)
+    rowptr_h, colidx_h, w_h = host_csr(tiny)
+    for _ in range(2):
+        out.fill_(float("nan")); dH.fill_(float("nan"))
+        g.dg_aggregate_host(H, G, binding.DG_OP_MEAN, out, dH, ws)
+        torch.cuda.synchronize()
+        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, H.numpy(), oracle.OP_MEAN)
+        assert_within_bound(out.numpy(), ref, mag, "host fwd")
+        ref, mag = oracle.ap_backward(rowptr_h, *csc, G.numpy(), oracle.OP_MEAN)
+        assert_within_bound(dH.numpy(), ref, mag, "host bwd")
+    # forward only
+    out.fill_(float("nan"))
+    g.dg_aggregate_host(H, None, binding.DG_OP_SUM, out, None, ws)
+    torch.cuda.synchronize()
+    ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, H.numpy(), oracle.OP_SUM)
+    assert_within_bound(out.numpy(), ref, mag, "host fwd only")
+
+
 # ------------------------------------------------------------------ mid-size workloads, in full
 @pytest.mark.parametrize("name,scale,F,ops", [
     ("reddit_like", 0.02, 602, (binding.DG_OP_MEAN,)),
