@@ -85,6 +85,24 @@ def compulsory_bytes(n, nnz, F, weighted, n_ref, inv_deg_gather):
     return b
 
 
+def max_over_ranks(x: float, world: int, device="cpu") -> float:
+    """Slowest rank's time: all-reduce(MAX) over the default process group (NCCL on GPUs, gloo in
+    the CPU tests); the identity for one rank."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_step: float, ms_per_step: float, world: int) -> float:
+    """Units all replicas processed per second: every rank runs the same workload (weak scaling)
+    and the step time is the slowest rank's."""
+    return world * units_per_step / (ms_per_step * 1e-3)
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -321,13 +339,10 @@ def main():
     if clocks is not None:
         clocks["remeasured"] = remeasured
         clocks["rejected"] = clocks_bad(clocks)
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
     units_per_step = 2 * sg.nnz * F                 # forward + backward edge*feature products
-    value = world * units_per_step / (ms_per_step * 1e-3)
+    value = whole_job_value(units_per_step, ms_per_step, world)
 
     # ---------------------------------------------------------------- roofline of the dominant kernel
     peak, peak_kind = measured_peaks()
@@ -413,12 +428,8 @@ def main():
         b.record(stream)
         torch.cuda.synchronize()
         e2e_ms = a.elapsed_time(b)
-        if world > 1:
-            t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_ms = float(t.item())
-        e2e_ms /= args.e2e_steps
-        e2e = {"value": world * units_per_step / (e2e_ms * 1e-3), "unit": UNIT,
+        e2e_ms = max_over_ranks(e2e_ms, world, dev) / args.e2e_steps
+        e2e = {"value": whole_job_value(units_per_step, e2e_ms, world), "unit": UNIT,
                "h2d_bytes_per_step": 2 * sg.n * F * 4, "d2h_bytes_per_step": 2 * sg.n * F * 4,
                "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                "call": "dg_aggregate_host (pinned host H, dOut in; out, dH back)"}
