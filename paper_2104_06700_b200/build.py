@@ -33,7 +33,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB_PATH
     nvcc = os.environ.get("NVCC", "nvcc")
     flags = [f for f in NVCC_FLAGS if not f.startswith("--use_fast_math")]
-    flags += os.environ.get("DG_NVCC_EXTRA", "").split()
     if verbose:
         flags += ["-Xptxas", "-v"]
     objs = []

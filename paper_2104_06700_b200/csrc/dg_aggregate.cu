@@ -1,8 +1,8 @@
 // Aggregation kernels: out[r] = rs_r * sum_k s_k * X[idx[k]] over one segment of a CSR (forward)
 // or CSC (backward) structure.  This is the pull loop of Algorithm 1 of the paper; the register
-// accumulation with one store per row follows the idea of Algorithm 3, and the split of the
-// feature dimension into slices that keep the gathered matrix L2-resident plays the role that
-// source blocking (Algorithm 2) plays on a CPU cache.
+// accumulation with one store per row follows the idea of Algorithm 3, and cutting the source
+// vertices into blocks whose rows of X stay L2-resident is Algorithm 2 with L2 in the role of
+// the CPU cache (one launch per block, later launches adding to the output).
 //
 // Work decomposition
 //   light segments (length <= heavy_threshold): every warp owns rows_per_warp consecutive
@@ -12,9 +12,10 @@
 //     needs fewer than 32 vectors the warp is cut into groups of G lanes and the groups take
 //     different edges of the same segment; their partial sums are combined by a fixed shuffle
 //     tree.  U load steps per lane are in flight before the first add.
-//   heavy segments: one thread block per segment (the first blocks of the same launch loop over
-//     the heavy list); the 8 warps take interleaved batches of 32 edges and combine in shared
-//     memory in warp order.
+//   heavy segments: one thread block per segment; the first blocks of the same launch (as many
+//     as the device keeps resident) loop over the heavy list, which is ordered longest first;
+//     the 8 warps take interleaved batches of 32 edges and combine in shared memory in warp
+//     order.
 // Every output element is produced by one thread in an order fixed by the launch shape, so the
 // result is deterministic and needs no atomics in either direction.
 #include "dg_internal.cuh"
@@ -97,15 +98,12 @@ __device__ __forceinline__ void load_batch(const ApArgs& a, int64_t b, int end, 
   }
 }
 
-#ifndef DG_U_CPL1
-#define DG_U_CPL1 8
-#endif
 template <int VEC, int G, int CPL>
 struct Shape {
   static constexpr int NG = 32 / G;  // edges one warp-wide load instruction covers
   // load steps in flight per lane (fewer when a step is several vectors wide), and no more
   // steps than one 32-edge batch holds
-  static constexpr int U0 = CPL == 1 ? DG_U_CPL1 : (CPL == 2 ? 4 : (VEC <= 2 ? 4 : 2));
+  static constexpr int U0 = CPL == 1 ? 8 : (CPL == 2 ? 4 : (VEC <= 2 ? 4 : 2));
   static constexpr int U = (U0 * NG > 32) ? (32 / NG) : U0;
 };
 
