@@ -59,6 +59,9 @@ def parse_args():
     ap.add_argument("--cpu-seconds", type=float, default=15.0,
                     help="target CPU time of the oracle sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sorted-ids", action="store_true",
+                    help="keep the generator's construction order of vertex ids (communities "
+                         "contiguous) instead of a random permutation; reported separately")
     ap.add_argument("--set", action="append", default=[],
                     help="library knob name=value (heavy_threshold, slice_features, rows_per_block)")
     return ap.parse_args()
@@ -242,7 +245,8 @@ def main():
     op_code = binding.DG_OP_MEAN if op == "mean" else binding.DG_OP_SUM
 
     # ---------------------------------------------------------------- inputs (seeded, synthetic)
-    sg = synth.make(args.workload, device=dev, scale=args.scale)
+    extra = {"sorted_ids": True} if args.sorted_ids else {}
+    sg = synth.make(args.workload, device=dev, scale=args.scale, **extra)
     torch.cuda.empty_cache()
     F = args.feat or sg.F
     weighted = sg.edge_w is not None
@@ -463,7 +467,7 @@ def main():
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
                        "F": F, "op": op, "weighted": weighted, "step": "fwd AP + bwd AP",
-                       "replicas": world,
+                       "replicas": world, "sorted_ids": bool(args.sorted_ids),
                        "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
                        else "H, out, dOut, dH separate", "l2": "inputs larger than L2 (no flush needed)"
                        if sg.n * F * 4 > 252e6 else "inputs fit L2: warm-L2 numbers",

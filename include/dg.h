@@ -177,7 +177,8 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *                      before the launch turns to the light rows; 0 = as many as are resident
  *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
- *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows)
+ *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows;
+ *                      0 = about 1024 edges per warp, between 32 and 248 rows per block)
  *   "l2_budget_mb"     MiB of the gathered matrix one launch may keep L2-resident
  *   "source_blocks"    number of source-vertex ranges the pass is cut into, one launch each
  *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,

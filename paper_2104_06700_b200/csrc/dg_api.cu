@@ -62,9 +62,21 @@ static dg_status_t refresh_heavy(Graph* g, bool csr, bool csc, cudaStream_t s) {
   return DG_OK;
 }
 
-// rows_per_block is rounded up to a whole number of rows per warp (8 warps per block).
+// rows_per_block is rounded up to a whole number of rows per warp (8 warps per block).  0 picks
+// about 1024 edges per warp, between 4 and 31 rows: short rows want long-lived blocks (less
+// block turnover), long rows want many blocks.
 static int32_t rows_per_warp(const Graph* g) {
-  int64_t r = (g->rows_per_block + 7) / 8;
+  int64_t r;
+  if (g->rows_per_block > 0) {
+    r = (g->rows_per_block + 7) / 8;
+  } else {
+    const double avg = g->n > 0 ? (double)g->nnz / (double)g->n : 1.0;
+    r = (int64_t)(1024.0 / (avg > 1.0 ? avg : 1.0));
+    if (r < 4) r = 4;
+    // small graphs: keep at least 64 warps' worth of row runs per SM
+    const int64_t fill = g->n / ((int64_t)g->sm_count * 64);
+    if (r > fill) r = fill;
+  }
   return (int32_t)(r < 1 ? 1 : (r > 31 ? 31 : r));
 }
 
@@ -373,7 +385,7 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     return DG_OK;
   }
   if (!strcmp(name, "rows_per_block")) {
-    if (value < 1 || value > 248) return invalid("rows_per_block must be in [1, 248]");
+    if (value < 0 || value > 248) return invalid("rows_per_block must be in [0, 248]");
     g->rows_per_block = value;
     return DG_OK;
   }

@@ -49,7 +49,7 @@ struct dg_graph {
   int64_t heavy_threshold = 1024;
   int64_t heavy_built_for = 0;   // threshold the heavy lists were built with
   int64_t slice_features = 0;    // 0 = automatic
-  int64_t rows_per_block = 32;
+  int64_t rows_per_block = 0;    // 0 = from the average row length
   int64_t heavy_blocks_per_sm = 0;  // blocks per SM that walk the heavy list; 0 = all resident ones
   int64_t l2_budget_bytes = 0;   // bytes of the gathered matrix one launch may keep L2-resident
   int64_t source_blocks = 0;     // 0 = automatic, else 1, 2, 4, 8 or 16
