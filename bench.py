@@ -364,7 +364,8 @@ def main():
         traffic = t[dom] / per_call
     roofline = {
         "bound": "hbm",
-        "kernel": f"ap_kernel ({dom}: {per_call} launch(es) per dg_aggregate_{dom} call)",
+        "kernel": ("ap_kernel_r48" if (weighted or (dom == "bwd" and op == "mean")) and F >= 64
+                   else "ap_kernel") + f" ({dom}: {per_call} launch(es) per dg_aggregate_{dom} call)",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_kind": f"of {peak_kind}", "frac_of_north_star_8TBs": achieved / NORTH_STAR_HBM_GBS,
         "launches_per_call": per_call,
