@@ -35,11 +35,11 @@ NORTH_STAR_HBM_GBS = 8000.0
 # summed over its launches, from the ncu captures summarised under profiles/.  Reported as
 # roofline.traffic only while the library still has the version the capture was taken with.
 NCU_TRAFFIC = {
-    ("reddit_like", 602, "mean", 1.0): {"version": "libdgagg 0.4 sm_100a", "fwd": 8.4235e9, "bwd": 11.5795e9},
-    ("products_like", 100, "mean", 1.0): {"version": "libdgagg 0.4 sm_100a", "fwd": 30.962e9, "bwd": 32.117e9},
-    ("papers_like", 128, "sum", 0.1): {"version": "libdgagg 0.4 sm_100a", "fwd": 28.194e9, "bwd": 74.177e9},
+    ("reddit_like", 602, "mean", 1.0): {"version": "libdgagg 0.5 sm_100a", "fwd": 8.421e9, "bwd": 11.682e9},
+    ("products_like", 100, "mean", 1.0): {"version": "libdgagg 0.5 sm_100a", "fwd": 31.024e9, "bwd": 32.159e9},
+    ("papers_like", 128, "sum", 0.1): {"version": "libdgagg 0.5 sm_100a", "fwd": 28.556e9, "bwd": 74.214e9},
     # full size is too large to capture: the scale-0.1 capture times 10 (edges and rows both x10)
-    ("papers_like", 128, "sum", 1.0): {"version": "libdgagg 0.4 sm_100a", "fwd": 281.94e9, "bwd": 741.77e9},
+    ("papers_like", 128, "sum", 1.0): {"version": "libdgagg 0.5 sm_100a", "fwd": 285.56e9, "bwd": 742.14e9},
 }
 
 

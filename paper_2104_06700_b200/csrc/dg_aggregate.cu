@@ -111,10 +111,10 @@ struct Shape {
 // into acc.  Lane group `grp` takes edges s+grp, s+grp+NG, ...  Full steps of U*NG edges run
 // without predicates; the ragged end runs once with predicated loads.  xrow[c] is the address
 // of this lane's c-th vector inside row 0 of X.
-template <int VEC, int G, int CPL, bool SCALED>
+template <int VEC, int G, int CPL, bool SCALED, bool STAGE>
 __device__ __forceinline__ void add_edges(const char* const (&xrow)[CPL], uint32_t row_bytes,
                                           int32_t cur_u, float cur_s, int s, int e, int grp,
-                                          typename Vec<VEC>::T (&acc)[CPL]) {
+                                          typename Vec<VEC>::T (&acc)[CPL], uint2* stage) {
   using V = typename Vec<VEC>::T;
   constexpr int NG = Shape<VEC, G, CPL>::NG;
   constexpr int U = Shape<VEC, G, CPL>::U;
@@ -123,14 +123,33 @@ __device__ __forceinline__ void add_edges(const char* const (&xrow)[CPL], uint32
   // that they hold no registers during the loads: that regime lives on occupancy.  With wider
   // lanes (4 or 2 steps) they are fetched with the loads and the adds do not wait for a shuffle.
   constexpr bool kLate = CPL == 1;
+  // Scaled, wide lanes, source-blocked (L2-resident) passes: the batch's (id, factor) pairs go
+  // through shared memory, so that one 8-byte broadcast load per step replaces two shuffles:
+  // fewer wavefronts on the load/store pipe, which is what bounds that case (Reddit-like
+  // backward 20.0 -> 19.3 ms).  Passes with short row pieces lose more on the extra store and
+  // warp barriers per call than they gain (Products-like F = 256: 14.0 -> 16.0 ms), so the
+  // passes without source blocks keep the shuffles.
+  constexpr bool kStaged = SCALED && !kLate && STAGE;
+  if (kStaged) {
+    __syncwarp();
+    stage[threadIdx.x & 31] = make_uint2((uint32_t)cur_u, __float_as_uint(cur_s));
+    __syncwarp();
+  }
   for (; p + U * NG <= e; p += U * NG) {
     V v[U][CPL];
     float sc[kLate ? 1 : U];
 #pragma unroll
     for (int j = 0; j < U; ++j) {
       const int src = p + j * NG + grp;
-      const uint32_t u = (uint32_t)__shfl_sync(kFull, cur_u, src);
-      if (SCALED && !kLate) sc[j] = __shfl_sync(kFull, cur_s, src);
+      uint32_t u;
+      if (kStaged) {
+        const uint2 us = stage[src];
+        u = us.x;
+        sc[j] = __uint_as_float(us.y);
+      } else {
+        u = (uint32_t)__shfl_sync(kFull, cur_u, src);
+        if (SCALED && !kLate) sc[j] = __shfl_sync(kFull, cur_s, src);
+      }
       const uint64_t off = (uint64_t)u * row_bytes;
 #pragma unroll
       for (int c = 0; c < CPL; ++c) v[j][c] = ldg_vec(xrow[c] + off, V());
@@ -190,6 +209,8 @@ template <int VEC, int G, int CPL, bool SCALED, bool SEG>
 __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_blocks,
                                            float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
   using V = typename Vec<VEC>::T;
+  __shared__ uint2 stage_heavy[kWarpsPerBlock][32];
+  uint2* stage = stage_heavy[threadIdx.x >> 5];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int grp = lane / G;
@@ -223,7 +244,8 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_bloc
     while (b < hi) {
       const bool more = hi - b > kBlock;
       if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
-      add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
+      add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
+                                     stage);
       if (!more) break;
       b += kBlock;
       cur_u = nxt_u;
@@ -258,6 +280,8 @@ template <int VEC, int G, int CPL, bool SCALED, bool SEG>
 __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
                                         float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
   using V = typename Vec<VEC>::T;
+  __shared__ uint2 stage_light[kWarpsPerBlock][32];
+  uint2* stage = stage_light[threadIdx.x >> 5];
   const int lane = threadIdx.x & 31;
   const int warp = threadIdx.x >> 5;
   const int grp = lane / G;
@@ -344,7 +368,8 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
 #pragma unroll
       for (int c = 0; c < CPL; ++c) zero(acc[c]);
       for (int b = lo; b < hi; b += 32) {
-        add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc);
+        add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
+                                     stage);
         cur_u = nxt_u;
         cur_s = nxt_s;
         if (qi < 32) {
@@ -396,7 +421,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
           load_batch<SCALED>(a, (int64_t)b + 32, stream_end, lane, nxt_u, nxt_s);
         }
         const int e = min(hi - b, 32);
-        add_edges<VEC, G, CPL, SCALED>(xrow, row_bytes, cur_u, cur_s, p - b, e, grp, acc);
+        add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, p - b, e, grp, acc, stage);
         p = b + e;
       }
       combine_groups<VEC, G, CPL>(acc);
