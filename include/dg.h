@@ -18,7 +18,11 @@
  *     legacy default stream.  Calls that take a stream only enqueue work on it;
  *   - feature matrices are dense, row-major, fp32, leading dimension F, 1 <= F <= 2^20;
  *   - rowptr/colptr are int64, vertex ids are int32 (n < 2^31), nnz < 2^31;
- *   - no call aborts, traps or waits without bound on the device.
+ *   - no call aborts, traps or waits without bound on the device;
+ *   - a handle may be used from any thread, by one thread at a time; different handles are
+ *     independent.  Calls on one handle that are queued on different streams are not ordered
+ *     against each other by the library (source-blocked passes read what the previous launch
+ *     of the same call wrote, so one call's launches all go to the stream it was given).
  */
 #ifndef DG_H_
 #define DG_H_

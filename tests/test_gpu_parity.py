@@ -224,6 +224,41 @@ def test_source_blocking_weighted_and_unsorted_rows():
             check_fwd_bwd(g, (rowptr, cols, w), H, G, op, csc)
 
 
+def test_deterministic_bits_with_source_blocks_and_heavy_rows():
+    """Same call, same data, same bits: also when the pass is cut into source blocks (later
+    launches add to the output) and some rows take the block-per-row path."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.02)
+    g = make_graph(sg)
+    g.dg_graph_set_param("source_blocks", 4)
+    g.dg_graph_set_param("heavy_threshold", 128)
+    g.dg_graph_transpose()
+    H = synth.features(sg.n, 602, 3, DEV)
+    for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+        a = g.dg_aggregate_fwd(H, op).clone()
+        b = g.dg_aggregate_bwd(H, op).clone()
+        for _ in range(3):
+            assert torch.equal(a, g.dg_aggregate_fwd(H, op))
+            assert torch.equal(b, g.dg_aggregate_bwd(H, op))
+
+
+def test_feature_width_limit_and_parameter_ranges(tiny):
+    g = make_graph(tiny)
+    lib = binding.lib()
+    import ctypes
+    H = synth.features(tiny.n, 4, 1, DEV)
+    st = lib.dg_aggregate_fwd(g._h, ctypes.c_void_p(H.data_ptr()), (1 << 20) + 4, 0,
+                              ctypes.c_void_p(H.data_ptr() + 64), None)
+    assert st == binding.DG_ERR_UNSUPPORTED
+    for name, bad in (("heavy_threshold", 1), ("rows_per_block", 249), ("source_blocks", 3),
+                      ("l2_budget_mb", 0), ("heavy_blocks_per_sm", 33), ("slice_features", -1)):
+        with pytest.raises(binding.DgError) as e:
+            g.dg_graph_set_param(name, bad)
+        assert e.value.status == binding.DG_ERR_INVALID_ARG
+    for name in ("heavy_threshold", "rows_per_block", "source_blocks", "l2_budget_mb",
+                 "heavy_blocks_per_sm", "slice_features"):
+        g.dg_graph_get_param(name)
+
+
 # ------------------------------------------------------------------ errors never trap
 def test_error_statuses(tiny):
     g = make_graph(tiny)
