@@ -60,7 +60,8 @@ typedef struct dg_graph* dg_graph_t;
  *           edge and broadcast over the F features), or NULL for the unary copy of Eq. 2
  * The handle BORROWS the three arrays: they must stay valid and unchanged until
  * dg_graph_destroy.  The call allocates a few small device arrays that it owns (1/in-degree
- * per vertex, the lists of heavy rows) and synchronises the device once.
+ * per vertex, the lists of heavy rows and, for graphs with at least 64 edges per vertex, 17
+ * int32 split pointers per vertex for source blocking) and synchronises the device once.
  * The arrays are trusted; dg_graph_validate checks them.
  */
 dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
