@@ -157,6 +157,19 @@ dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t
                              void* stream);
 
 /*
+ * The same two passes with the gathered matrix stored as bf16 (two bytes per element, the
+ * upper half of an fp32; the paper's Conclusion names reduced precision as future work).  Every
+ * gathered byte is halved; products and sums are fp32 (a bf16 value converts to fp32 exactly)
+ * and the output is fp32, so the result equals the fp32 entry point's on the same values and
+ * the same error bound holds.  F must be even (16-byte loads need F % 8 == 0 and a 16-byte
+ * aligned H; narrower loads are used otherwise); DG_ERR_UNSUPPORTED for an odd F.
+ */
+dg_status_t dg_aggregate_fwd_bf16(dg_graph_t g, const uint16_t* H, int32_t F, dg_op_t op,
+                                  float* out, void* stream);
+dg_status_t dg_aggregate_bwd_bf16(dg_graph_t g, const uint16_t* dOut, int32_t F, dg_op_t op,
+                                  float* dH, void* stream);
+
+/*
  * Forward and backward AP with the feature matrices in HOST memory (pinned memory makes the
  * copies asynchronous and lets them overlap the kernels; pageable memory works but serialises).
  * Computes what dg_aggregate_fwd on H_host and dg_aggregate_bwd on dOut_host compute and leaves

@@ -26,6 +26,7 @@ DG_OP_MEAN = 1
 EXPORTS = [
     "dg_graph_create", "dg_graph_destroy", "dg_graph_validate", "dg_graph_transpose_workspace",
     "dg_graph_transpose", "dg_graph_transpose_static", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
+    "dg_aggregate_fwd_bf16", "dg_aggregate_bwd_bf16",
     "dg_aggregate_host_workspace", "dg_aggregate_host", "dg_graph_set_param",
     "dg_graph_get_param", "dg_kernel_launch_count", "dg_last_error", "dg_version",
 ]
@@ -61,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.dg_graph_get_csc.argtypes = [p, pp, pp, pp, pp]
         L.dg_aggregate_fwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_bwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
+        L.dg_aggregate_fwd_bf16.argtypes = [p, p, i32, ctypes.c_int, p, p]
+        L.dg_aggregate_bwd_bf16.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_host_workspace.argtypes = [p, i32]
         L.dg_aggregate_host_workspace.restype = sz
         L.dg_aggregate_host.argtypes = [p, p, p, i32, ctypes.c_int, p, p, p, sz, p]
@@ -215,6 +218,26 @@ class Graph:
             dH = torch.empty_like(dOut)
         _check(lib().dg_aggregate_bwd(self._h, _dev_ptr(dOut, torch.float32, "dOut"), F, int(op),
                                       _dev_ptr(dH, torch.float32, "dH"), _stream(stream)))
+        return dH
+
+    def dg_aggregate_fwd_bf16(self, H: torch.Tensor, op: int, out: Optional[torch.Tensor] = None,
+                              stream=None) -> torch.Tensor:
+        """H is a torch.bfloat16 matrix; the result is fp32."""
+        F = H.shape[1]
+        if out is None:
+            out = torch.empty(H.shape, dtype=torch.float32, device=H.device)
+        _check(lib().dg_aggregate_fwd_bf16(self._h, _dev_ptr(H, torch.bfloat16, "H"), F, int(op),
+                                           _dev_ptr(out, torch.float32, "out"), _stream(stream)))
+        return out
+
+    def dg_aggregate_bwd_bf16(self, dOut: torch.Tensor, op: int,
+                              dH: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        F = dOut.shape[1]
+        if dH is None:
+            dH = torch.empty(dOut.shape, dtype=torch.float32, device=dOut.device)
+        _check(lib().dg_aggregate_bwd_bf16(self._h, _dev_ptr(dOut, torch.bfloat16, "dOut"), F,
+                                           int(op), _dev_ptr(dH, torch.float32, "dH"),
+                                           _stream(stream)))
         return dH
 
     def dg_aggregate_host_workspace(self, F: int) -> int:

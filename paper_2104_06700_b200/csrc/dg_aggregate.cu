@@ -27,10 +27,22 @@ constexpr int kWarpsPerBlock = 8;
 constexpr int kBlock = kWarpsPerBlock * 32;
 constexpr unsigned kFull = 0xffffffffu;
 
+// Accumulators are fp32 vectors of VEC floats; f8 is the 8-wide one (two float4).
+struct f8 { float4 lo, hi; };
 template <int VEC> struct Vec;
 template <> struct Vec<1> { using T = float; };
 template <> struct Vec<2> { using T = float2; };
 template <> struct Vec<4> { using T = float4; };
+template <> struct Vec<8> { using T = f8; };
+
+// Storage type of the gathered matrix: fp32, or bf16 (NEXT: halves every gathered byte; the sums
+// stay fp32).  Pack<E, VEC>::Load is what one lane loads for VEC consecutive elements.
+struct F32 { static constexpr int kBytes = 4; };
+struct BF16 { static constexpr int kBytes = 2; };
+template <typename E, int VEC> struct Pack { using Load = typename Vec<VEC>::T; };
+template <> struct Pack<BF16, 2> { using Load = uint32_t; };
+template <> struct Pack<BF16, 4> { using Load = uint2; };
+template <> struct Pack<BF16, 8> { using Load = uint4; };
 
 __device__ __forceinline__ float ldg_vec(const char* p, float) {
   return __ldg(reinterpret_cast<const float*>(p));
@@ -41,6 +53,18 @@ __device__ __forceinline__ float2 ldg_vec(const char* p, float2) {
 __device__ __forceinline__ float4 ldg_vec(const char* p, float4) {
   return __ldg(reinterpret_cast<const float4*>(p));
 }
+__device__ __forceinline__ uint32_t ldg_vec(const char* p, uint32_t) {
+  return __ldg(reinterpret_cast<const uint32_t*>(p));
+}
+__device__ __forceinline__ uint2 ldg_vec(const char* p, uint2) {
+  return __ldg(reinterpret_cast<const uint2*>(p));
+}
+__device__ __forceinline__ uint4 ldg_vec(const char* p, uint4) {
+  return __ldg(reinterpret_cast<const uint4*>(p));
+}
+// a 32-bit word holds two bf16 values: the low half is the element with the lower index
+__device__ __forceinline__ float bf_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
 __device__ __forceinline__ float ld_vec(const float* p, float) { return *p; }
 __device__ __forceinline__ float2 ld_vec(const float* p, float2) {
   return *reinterpret_cast<const float2*>(p);
@@ -48,6 +72,15 @@ __device__ __forceinline__ float2 ld_vec(const float* p, float2) {
 __device__ __forceinline__ float4 ld_vec(const float* p, float4) {
   return *reinterpret_cast<const float4*>(p);
 }
+__device__ __forceinline__ f8 ld_vec(const float* p, f8) {
+  f8 v;
+  v.lo = *reinterpret_cast<const float4*>(p);
+  v.hi = *reinterpret_cast<const float4*>(p + 4);
+  return v;
+}
+__device__ __forceinline__ void zero(uint32_t& a) { a = 0u; }
+__device__ __forceinline__ void zero(uint2& a) { a.x = a.y = 0u; }
+__device__ __forceinline__ void zero(uint4& a) { a.x = a.y = a.z = a.w = 0u; }
 __device__ __forceinline__ void zero(float& a) { a = 0.f; }
 __device__ __forceinline__ void zero(float2& a) { a.x = a.y = 0.f; }
 __device__ __forceinline__ void zero(float4& a) { a.x = a.y = a.z = a.w = 0.f; }
@@ -55,6 +88,28 @@ __device__ __forceinline__ void add(float& a, const float& v) { a += v; }
 __device__ __forceinline__ void add(float2& a, const float2& v) { a.x += v.x; a.y += v.y; }
 __device__ __forceinline__ void add(float4& a, const float4& v) {
   a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+}
+__device__ __forceinline__ void zero(f8& a) { zero(a.lo); zero(a.hi); }
+__device__ __forceinline__ void add(f8& a, const f8& v) { add(a.lo, v.lo); add(a.hi, v.hi); }
+// packed bf16 loads into fp32 accumulators
+__device__ __forceinline__ void add(float2& a, uint32_t v) { a.x += bf_lo(v); a.y += bf_hi(v); }
+__device__ __forceinline__ void add(float4& a, uint2 v) {
+  a.x += bf_lo(v.x); a.y += bf_hi(v.x); a.z += bf_lo(v.y); a.w += bf_hi(v.y);
+}
+__device__ __forceinline__ void add(f8& a, uint4 v) {
+  add(a.lo, make_uint2(v.x, v.y));
+  add(a.hi, make_uint2(v.z, v.w));
+}
+__device__ __forceinline__ void fma(float2& a, float s, uint32_t v) {
+  a.x = fmaf(s, bf_lo(v), a.x); a.y = fmaf(s, bf_hi(v), a.y);
+}
+__device__ __forceinline__ void fma(float4& a, float s, uint2 v) {
+  a.x = fmaf(s, bf_lo(v.x), a.x); a.y = fmaf(s, bf_hi(v.x), a.y);
+  a.z = fmaf(s, bf_lo(v.y), a.z); a.w = fmaf(s, bf_hi(v.y), a.w);
+}
+__device__ __forceinline__ void fma(f8& a, float s, uint4 v) {
+  fma(a.lo, s, make_uint2(v.x, v.y));
+  fma(a.hi, s, make_uint2(v.z, v.w));
 }
 __device__ __forceinline__ void fma(float& a, float s, const float& v) { a = fmaf(s, v, a); }
 __device__ __forceinline__ void fma(float2& a, float s, const float2& v) {
@@ -67,6 +122,7 @@ __device__ __forceinline__ void fma(float4& a, float s, const float4& v) {
 __device__ __forceinline__ void scale(float& a, float s) { a *= s; }
 __device__ __forceinline__ void scale(float2& a, float s) { a.x *= s; a.y *= s; }
 __device__ __forceinline__ void scale(float4& a, float s) { a.x *= s; a.y *= s; a.z *= s; a.w *= s; }
+__device__ __forceinline__ void scale(f8& a, float s) { scale(a.lo, s); scale(a.hi, s); }
 __device__ __forceinline__ float shfl_xor(float a, int m) { return __shfl_xor_sync(kFull, a, m); }
 __device__ __forceinline__ float2 shfl_xor(float2 a, int m) {
   return make_float2(__shfl_xor_sync(kFull, a.x, m), __shfl_xor_sync(kFull, a.y, m));
@@ -75,9 +131,23 @@ __device__ __forceinline__ float4 shfl_xor(float4 a, int m) {
   return make_float4(__shfl_xor_sync(kFull, a.x, m), __shfl_xor_sync(kFull, a.y, m),
                      __shfl_xor_sync(kFull, a.z, m), __shfl_xor_sync(kFull, a.w, m));
 }
+__device__ __forceinline__ f8 shfl_xor(f8 a, int m) {
+  f8 r;
+  r.lo = shfl_xor(a.lo, m);
+  r.hi = shfl_xor(a.hi, m);
+  return r;
+}
 __device__ __forceinline__ void stcs_vec(float* p, float v) { __stcs(p, v); }
 __device__ __forceinline__ void stcs_vec(float* p, float2 v) { __stcs(reinterpret_cast<float2*>(p), v); }
 __device__ __forceinline__ void stcs_vec(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+__device__ __forceinline__ void stcs_vec(float* p, f8 v) {
+  __stcs(reinterpret_cast<float4*>(p), v.lo);
+  __stcs(reinterpret_cast<float4*>(p + 4), v.hi);
+}
+__device__ __forceinline__ void st_smem(float* p, f8 v) {
+  p[0] = v.lo.x; p[1] = v.lo.y; p[2] = v.lo.z; p[3] = v.lo.w;
+  p[4] = v.hi.x; p[5] = v.hi.y; p[6] = v.hi.z; p[7] = v.hi.w;
+}
 __device__ __forceinline__ void st_smem(float* p, float v) { p[0] = v; }
 __device__ __forceinline__ void st_smem(float* p, float2 v) { p[0] = v.x; p[1] = v.y; }
 __device__ __forceinline__ void st_smem(float* p, float4 v) {
@@ -111,11 +181,11 @@ struct Shape {
 // into acc.  Lane group `grp` takes edges s+grp, s+grp+NG, ...  Full steps of U*NG edges run
 // without predicates; the ragged end runs once with predicated loads.  xrow[c] is the address
 // of this lane's c-th vector inside row 0 of X.
-template <int VEC, int G, int CPL, bool SCALED, bool STAGE>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool STAGE>
 __device__ __forceinline__ void add_edges(const char* const (&xrow)[CPL], uint32_t row_bytes,
                                           int32_t cur_u, float cur_s, int s, int e, int grp,
                                           typename Vec<VEC>::T (&acc)[CPL], uint2* stage) {
-  using V = typename Vec<VEC>::T;
+  using V = typename Pack<E, VEC>::Load;  // as loaded; unpacked while adding
   constexpr int NG = Shape<VEC, G, CPL>::NG;
   constexpr int U = Shape<VEC, G, CPL>::U;
   int p = s;
@@ -205,7 +275,7 @@ __device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL])
 // Block-per-row path for the heavy segments: block x of the first `heavy_blocks` blocks takes
 // entries x, x + heavy_blocks, ... of the heavy list; its 8 warps sum interleaved 32-edge
 // batches and the partial sums are combined in shared memory in warp order.
-template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
 __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_blocks,
                                            float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
   using V = typename Vec<VEC>::T;
@@ -218,14 +288,14 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_bloc
   const int f0 = blockIdx.y * a.slice_f;
   const int width = min(a.F, f0 + a.slice_f) - f0;
   const int chunks = width / VEC;
-  const uint32_t row_bytes = (uint32_t)a.F * 4u;
+  const uint32_t row_bytes = (uint32_t)a.F * (uint32_t)E::kBytes;
   const char* xrow[CPL];
   bool cok[CPL];
 #pragma unroll
   for (int c = 0; c < CPL; ++c) {
     const int ci = c0 + c * G;
     cok[c] = ci < chunks;
-    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * 4u;
+    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * E::kBytes;
   }
   const int count = min(*a.heavy_count, a.heavy_cap);
   for (int i = blockIdx.x; i < count; i += heavy_blocks) {
@@ -244,7 +314,7 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_bloc
     while (b < hi) {
       const bool more = hi - b > kBlock;
       if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
-      add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
+      add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
       if (!more) break;
       b += kBlock;
@@ -276,7 +346,7 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const int heavy_bloc
 // first, so the long segments start early); in the remaining blocks every warp owns
 // rows_per_warp consecutive light segments and streams their indices as one run of 32-edge
 // batches, the next batch always in flight while the current one is summed.
-template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
 __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
                                         float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
   using V = typename Vec<VEC>::T;
@@ -290,7 +360,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
   const int fend = min(a.F, f0 + a.slice_f);
   const int width = fend - f0;
   const int chunks = width / VEC;
-  const uint32_t row_bytes = (uint32_t)a.F * 4u;
+  const uint32_t row_bytes = (uint32_t)a.F * (uint32_t)E::kBytes;
 
   // Lanes whose vector falls beyond the slice re-read vector 0 and never store: the summing
   // loop then needs no per-lane predicate.
@@ -300,7 +370,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
   for (int c = 0; c < CPL; ++c) {
     const int ci = c0 + c * G;
     cok[c] = ci < chunks;
-    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * 4u;
+    xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * E::kBytes;
   }
 
   // Writes one finished row: scales by 1/length for the mean and, in a later source block, adds
@@ -368,7 +438,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
 #pragma unroll
       for (int c = 0; c < CPL; ++c) zero(acc[c]);
       for (int b = lo; b < hi; b += 32) {
-        add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
+        add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
         cur_u = nxt_u;
         cur_s = nxt_s;
@@ -421,7 +491,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
           load_batch<SCALED>(a, (int64_t)b + 32, stream_end, lane, nxt_u, nxt_s);
         }
         const int e = min(hi - b, 32);
-        add_edges<VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, p - b, e, grp, acc, stage);
+        add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, p - b, e, grp, acc, stage);
         p = b + e;
       }
       combine_groups<VEC, G, CPL>(acc);
@@ -430,13 +500,13 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const int heavy_blocks,
     return;
   }
 
-  heavy_rows<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+  heavy_rows<E, VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
 
-template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
 __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
 
 // The same kernel compiled for five resident blocks per SM (at most 48 registers).  The scaled
@@ -444,10 +514,10 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
 // else and would take 60 registers; measured on B200 the higher occupancy wins for them
 // (Reddit-like backward 22.0 -> 19.3 ms, Products-like backward 7.0 -> 6.2 ms), while the same
 // cap slows the unscaled variants down.
-template <int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
 __global__ void __launch_bounds__(kBlock, 5) ap_kernel_r48(const ApArgs a, const int heavy_blocks) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
 
 // Blocks that walk the heavy list: as many as the device keeps resident, so that the heavy
@@ -462,15 +532,16 @@ int heavy_block_count(const Graph* g, K kernel, size_t smem) {
   return g->sm_count * (per_sm < 1 ? 1 : per_sm);
 }
 
-template <int VEC, int G, int CPL, bool SCALED>
+template <typename E, int VEC, int G, int CPL, bool SCALED>
 dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
   if (a.n == 0) return DG_OK;
   void (*kernel)(const ApArgs, const int);
-  if constexpr (SCALED && VEC * CPL <= 4 && G >= 16) {
-    kernel = a.seg_lo ? ap_kernel_r48<VEC, G, CPL, SCALED, true>
-                      : ap_kernel_r48<VEC, G, CPL, SCALED, false>;
+  if constexpr (SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16) {
+    kernel = a.seg_lo ? ap_kernel_r48<E, VEC, G, CPL, SCALED, true>
+                      : ap_kernel_r48<E, VEC, G, CPL, SCALED, false>;
   } else {
-    kernel = a.seg_lo ? ap_kernel<VEC, G, CPL, SCALED, true> : ap_kernel<VEC, G, CPL, SCALED, false>;
+    kernel = a.seg_lo ? ap_kernel<E, VEC, G, CPL, SCALED, true>
+                      : ap_kernel<E, VEC, G, CPL, SCALED, false>;
   }
   const int heavy_blocks = heavy_block_count(g, kernel, 0);
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
@@ -482,43 +553,62 @@ dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_
   return DG_OK;
 }
 
-template <int VEC, bool SCALED>
+template <typename E, int VEC, bool SCALED>
 dg_status_t dispatch_shape(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
   const int chunks = (a.slice_f < a.F ? a.slice_f : a.F) / VEC;  // vectors per row slice
-  if (chunks <= 2) return launch_pair<VEC, 2, 1, SCALED>(g, a, slices, s);
-  if (chunks <= 4) return launch_pair<VEC, 4, 1, SCALED>(g, a, slices, s);
-  if (chunks <= 8) return launch_pair<VEC, 8, 1, SCALED>(g, a, slices, s);
-  if (chunks <= 16) return launch_pair<VEC, 16, 1, SCALED>(g, a, slices, s);
-  if (chunks <= 32) return launch_pair<VEC, 32, 1, SCALED>(g, a, slices, s);
-  if (chunks <= 64) return launch_pair<VEC, 32, 2, SCALED>(g, a, slices, s);
-  return launch_pair<VEC, 32, 4, SCALED>(g, a, slices, s);
+  if (chunks <= 2) return launch_pair<E, VEC, 2, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 4) return launch_pair<E, VEC, 4, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 8) return launch_pair<E, VEC, 8, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 16) return launch_pair<E, VEC, 16, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 32) return launch_pair<E, VEC, 32, 1, SCALED>(g, a, slices, s);
+  if (chunks <= 64) return launch_pair<E, VEC, 32, 2, SCALED>(g, a, slices, s);
+  return launch_pair<E, VEC, 32, 4, SCALED>(g, a, slices, s);
+}
+
+template <typename E, int VEC>
+dg_status_t dispatch_scaled(const Graph* g, const ApArgs& a, int slices, cudaStream_t s) {
+  return a.w ? dispatch_shape<E, VEC, true>(g, a, slices, s)
+             : dispatch_shape<E, VEC, false>(g, a, slices, s);
 }
 
 }  // namespace
 
-// Bytes of L2 one row slice of `slice` floats occupies: L2 allocates 128-byte lines, and a slice
-// that does not start on a line boundary in every row touches one more line.
-static double slice_footprint(int64_t F, int64_t slice) {
-  const int64_t bytes = slice * 4;
-  const bool aligned = (F * 4) % 128 == 0 && bytes % 128 == 0;
+// Bytes of L2 one row slice of `slice` elements of `eb` bytes occupies: L2 allocates 128-byte
+// lines, and a slice that does not start on a line boundary in every row touches one more line.
+static double slice_footprint(int64_t F, int64_t slice, int eb) {
+  const int64_t bytes = slice * eb;
+  const bool aligned = (F * eb) % 128 == 0 && bytes % 128 == 0;
   return (double)(((bytes + 127) / 128) * 128 + (aligned ? 0 : 128));
 }
 
 // Chooses the launch shape, then runs one launch per source block.
-//   vector width: the widest both matrices allow;
+//   vector width: the widest both matrices allow (16-byte loads of the gathered matrix when
+//     its rows and its base are 16-byte aligned, else 8 or 4 bytes);
 //   slice: at most 128 vectors per row slice (4 per lane);
 //   source blocks (Algorithm 2 of the paper, with L2 in the role of the CPU cache): when one
 //     slice of X over all n rows exceeds the L2 budget and the segments carry split pointers,
 //     the neighbour ids are cut into 2, 4, 8 or 16 ranges and each range is a launch of its
 //     own, so that the rows of X a launch gathers stay L2-resident; later launches add to Y.
-//     Without split pointers the slice is narrowed instead (down to 32 floats).
+//     Without split pointers the slice is narrowed instead (down to 128 bytes).
 dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split, cudaStream_t s) {
   ApArgs a = a0;
   if (a.n == 0) return DG_OK;
   const uintptr_t px = (uintptr_t)a.X, py = (uintptr_t)a.Y;
-  int vec = 1;
-  if (a.F % 4 == 0 && px % 16 == 0 && py % 16 == 0) vec = 4;
-  else if (a.F % 2 == 0 && px % 8 == 0 && py % 8 == 0) vec = 2;
+  const bool bf16 = a.x_bf16 != 0;
+  const int eb = bf16 ? 2 : 4;
+  int vec = 1;  // elements per lane and vector
+  if (bf16) {
+    if (a.F % 8 == 0 && px % 16 == 0 && py % 16 == 0) vec = 8;
+    else if (a.F % 4 == 0 && px % 8 == 0 && py % 16 == 0) vec = 4;
+    else if (a.F % 2 == 0 && px % 4 == 0 && py % 8 == 0) vec = 2;
+    else {
+      set_error("bf16 feature matrices need an even F and 4-byte (input) / 8-byte (output) alignment");
+      return DG_ERR_UNSUPPORTED;
+    }
+  } else {
+    if (a.F % 4 == 0 && px % 16 == 0 && py % 16 == 0) vec = 4;
+    else if (a.F % 2 == 0 && px % 8 == 0 && py % 8 == 0) vec = 2;
+  }
 
   const double budget = (double)g->l2_budget_bytes;
   const double avg_len = (double)g->nnz / (double)a.n;
@@ -529,7 +619,7 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
   int nb = 1;
   if (g->source_blocks > 0) {
     nb = split ? (int)g->source_blocks : 1;
-  } else if (g->slice_features <= 0 && (double)a.n * slice_footprint(a.F, slice) > budget) {
+  } else if (g->slice_features <= 0 && (double)a.n * slice_footprint(a.F, slice, eb) > budget) {
     if (split) {
       // widest slice first; a candidate is feasible when some block count keeps one block of
       // the slice inside the budget and leaves a row at least 32 edges per block on average
@@ -539,8 +629,9 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
         int64_t w = widths[t];
         if (w > slice) w = slice;
         int cand = 1;
-        while (cand < kFineBlocks && (double)a.n / cand * slice_footprint(a.F, w) > budget) cand *= 2;
-        if ((double)a.n / cand * slice_footprint(a.F, w) <= budget && avg_len / cand >= 32.0) {
+        while (cand < kFineBlocks && (double)a.n / cand * slice_footprint(a.F, w, eb) > budget)
+          cand *= 2;
+        if ((double)a.n / cand * slice_footprint(a.F, w, eb) <= budget && avg_len / cand >= 32.0) {
           slice = w;
           nb = cand;
           found = true;
@@ -552,8 +643,8 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
         if (slice > 8LL * vec) slice = 8LL * vec;
       }
     } else {
-      int64_t w = (int64_t)(budget / ((double)a.n * 4.0));
-      if (w >= 32) slice = w < slice ? w : slice;  // narrower than 128 bytes is not worth a pass
+      int64_t w = (int64_t)(budget / ((double)a.n * eb));
+      if (w * eb >= 128) slice = w < slice ? w : slice;  // under 128 bytes is not worth a pass
     }
   }
   slice = (slice / vec) * vec;
@@ -565,7 +656,6 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
   if (even <= slice) slice = even;
   a.slice_f = (int32_t)slice;
   const int slices = (int)((a.F + slice - 1) / slice);
-  const bool scaled = a.w != nullptr;
 
   const int per = kFineBlocks / nb;
   for (int j = 0; j < nb; ++j) {
@@ -575,9 +665,15 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
       a.accumulate = j > 0;
     }
     dg_status_t st;
-    if (vec == 4) st = scaled ? dispatch_shape<4, true>(g, a, slices, s) : dispatch_shape<4, false>(g, a, slices, s);
-    else if (vec == 2) st = scaled ? dispatch_shape<2, true>(g, a, slices, s) : dispatch_shape<2, false>(g, a, slices, s);
-    else st = scaled ? dispatch_shape<1, true>(g, a, slices, s) : dispatch_shape<1, false>(g, a, slices, s);
+    if (bf16) {
+      if (vec == 8) st = dispatch_scaled<BF16, 8>(g, a, slices, s);
+      else if (vec == 4) st = dispatch_scaled<BF16, 4>(g, a, slices, s);
+      else st = dispatch_scaled<BF16, 2>(g, a, slices, s);
+    } else {
+      if (vec == 4) st = dispatch_scaled<F32, 4>(g, a, slices, s);
+      else if (vec == 2) st = dispatch_scaled<F32, 2>(g, a, slices, s);
+      else st = dispatch_scaled<F32, 1>(g, a, slices, s);
+    }
     if (st != DG_OK) return st;
   }
   return DG_OK;

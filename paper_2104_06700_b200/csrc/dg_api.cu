@@ -80,8 +80,8 @@ static int32_t rows_per_warp(const Graph* g) {
   return (int32_t)(r < 1 ? 1 : (r > 31 ? 31 : r));
 }
 
-static dg_status_t check_features(const Graph* g, const float* in, float* out, int32_t F,
-                                  dg_op_t op) {
+static dg_status_t check_features(const Graph* g, const void* in, size_t in_elem_bytes, float* out,
+                                  int32_t F, dg_op_t op) {
   if (!g) return invalid("graph handle is NULL");
   if (F < 1) return invalid("F must be >= 1");
   if (F > (1 << 20)) {
@@ -91,10 +91,59 @@ static dg_status_t check_features(const Graph* g, const float* in, float* out, i
   if (op != DG_OP_SUM && op != DG_OP_MEAN) return invalid("op must be DG_OP_SUM or DG_OP_MEAN");
   if (g->n > 0) {
     if (!in || !out) return invalid("feature matrix pointer is NULL");
-    if (overlaps(in, out, (size_t)g->n * (size_t)F * sizeof(float)))
+    const size_t elems = (size_t)g->n * (size_t)F;
+    const uintptr_t x = (uintptr_t)in, y = (uintptr_t)out;
+    if (x < y + elems * sizeof(float) && y < x + elems * in_elem_bytes)
       return invalid("input and output feature matrices overlap");
   }
   return DG_OK;
+}
+
+// Forward / backward AP for either storage type of the gathered matrix.
+static dg_status_t run_forward(Graph* g, const void* H, bool bf16, int32_t F, dg_op_t op,
+                               float* out, void* stream) {
+  if (dg_status_t st = check_features(g, H, bf16 ? 2 : 4, out, F, op)) return st;
+  ApArgs a{};
+  a.ptr = g->rowptr;
+  a.idx = g->colidx;
+  a.w = g->edge_w;
+  a.X = H;
+  a.x_bf16 = bf16;
+  a.Y = out;
+  a.heavy_list = g->heavy_rows;
+  a.heavy_count = g->counters + 0;
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.n = g->n;
+  a.F = F;
+  a.mean_rows = op == DG_OP_MEAN;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
+  a.rows_per_warp = rows_per_warp(g);
+  return aggregate_run(g, a, g->split_csr, (cudaStream_t)stream);
+}
+
+static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F, dg_op_t op,
+                                float* dH, void* stream) {
+  if (dg_status_t st = check_features(g, dOut, bf16 ? 2 : 4, dH, F, op)) return st;
+  if (!g->transposed) {
+    set_error("the backward pass needs dg_graph_transpose first");
+    return DG_ERR_NOT_TRANSPOSED;
+  }
+  ApArgs a{};
+  a.ptr = g->colptr;
+  a.idx = g->rowidx_T;
+  a.w = op == DG_OP_MEAN ? g->mean_scale_T : g->w_T;
+  a.X = dOut;
+  a.x_bf16 = bf16;
+  a.Y = dH;
+  a.heavy_list = g->heavy_cols;
+  a.heavy_count = g->counters + 1;
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.n = g->n;
+  a.F = F;
+  a.mean_rows = 0;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
+  a.rows_per_warp = rows_per_warp(g);
+  return aggregate_run(g, a, g->split_csc, (cudaStream_t)stream);
 }
 
 }  // namespace dg
@@ -229,46 +278,22 @@ dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t
 
 dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op, float* out,
                              void* stream) {
-  if (dg_status_t st = check_features(g, H, out, F, op)) return st;
-  ApArgs a{};
-  a.ptr = g->rowptr;
-  a.idx = g->colidx;
-  a.w = g->edge_w;
-  a.X = H;
-  a.Y = out;
-  a.heavy_list = g->heavy_rows;
-  a.heavy_count = g->counters + 0;
-  a.heavy_cap = (int32_t)g->heavy_cap;
-  a.n = g->n;
-  a.F = F;
-  a.mean_rows = op == DG_OP_MEAN;
-  a.heavy_threshold = (int32_t)g->heavy_threshold;
-  a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, g->split_csr, (cudaStream_t)stream);
+  return run_forward(g, H, false, F, op, out, stream);
 }
 
 dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t op, float* dH,
                              void* stream) {
-  if (dg_status_t st = check_features(g, dOut, dH, F, op)) return st;
-  if (!g->transposed) {
-    set_error("dg_aggregate_bwd needs dg_graph_transpose first");
-    return DG_ERR_NOT_TRANSPOSED;
-  }
-  ApArgs a{};
-  a.ptr = g->colptr;
-  a.idx = g->rowidx_T;
-  a.w = op == DG_OP_MEAN ? g->mean_scale_T : g->w_T;
-  a.X = dOut;
-  a.Y = dH;
-  a.heavy_list = g->heavy_cols;
-  a.heavy_count = g->counters + 1;
-  a.heavy_cap = (int32_t)g->heavy_cap;
-  a.n = g->n;
-  a.F = F;
-  a.mean_rows = 0;
-  a.heavy_threshold = (int32_t)g->heavy_threshold;
-  a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, g->split_csc, (cudaStream_t)stream);
+  return run_backward(g, dOut, false, F, op, dH, stream);
+}
+
+dg_status_t dg_aggregate_fwd_bf16(dg_graph_t g, const uint16_t* H, int32_t F, dg_op_t op,
+                                  float* out, void* stream) {
+  return run_forward(g, H, true, F, op, out, stream);
+}
+
+dg_status_t dg_aggregate_bwd_bf16(dg_graph_t g, const uint16_t* dOut, int32_t F, dg_op_t op,
+                                  float* dH, void* stream) {
+  return run_backward(g, dOut, true, F, op, dH, stream);
 }
 
 size_t dg_aggregate_host_workspace(dg_graph_t g, int32_t F) {

@@ -69,7 +69,8 @@ struct ApArgs {
   const int64_t* ptr;         // n+1 segment pointers (rowptr or colptr)
   const int32_t* idx;         // neighbour ids (colidx or rowidx_T)
   const float* w;             // per-edge weight or nullptr
-  const float* X;             // n x F input
+  const void* X;              // n x F input: fp32, or bf16 when x_bf16 is set
+  int32_t x_bf16;
   float* Y;                   // n x F output
   const int32_t* heavy_list;  // segments longer than heavy_threshold
   const int32_t* heavy_count; // device scalar

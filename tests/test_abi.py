@@ -17,7 +17,7 @@ def libpath():
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "dg.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(dg_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(dg_[a-z0-9_]+)\s*\(", text)))
 
 
 def test_header_declares_the_call_list():
