@@ -58,6 +58,9 @@ def parse_args():
                     help="GraphSAGE epochs to time after 3 warm-up epochs (0 = skip)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0,
                     help="target CPU time of the oracle sample")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"],
+                    help="storage of the gathered matrices (sums and outputs are fp32 either "
+                         "way); bf16 is reported separately, the headline is f32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sorted-ids", action="store_true",
                     help="keep the generator's construction order of vertex ids (communities "
@@ -79,10 +82,10 @@ def measured_peaks():
     return 6650.0, "fallback"
 
 
-def compulsory_bytes(n, nnz, F, weighted, n_ref, inv_deg_gather):
+def compulsory_bytes(n, nnz, F, weighted, n_ref, inv_deg_gather, in_bytes=4):
     """Bytes one AP call must move once: pointers, indices, weights, the referenced rows of the
     input matrix read once, the output written once (+ the 1/deg vector for the mean backward)."""
-    b = (n + 1) * 8 + nnz * 4 + (nnz * 4 if weighted else 0) + n_ref * F * 4 + n * F * 4
+    b = (n + 1) * 8 + nnz * 4 + (nnz * 4 if weighted else 0) + n_ref * F * in_bytes + n * F * 4
     if inv_deg_gather:
         b += n * 4
     return b
@@ -286,6 +289,7 @@ def main():
     transpose_ms = e0.elapsed_time(e1)
     del scratch
     torch.cuda.empty_cache()
+    bf16 = args.dtype == "bf16"
     H = synth.features(sg.n, F, 100, dev)
     out = torch.empty_like(H)
     if two_buffers:
@@ -293,11 +297,17 @@ def main():
     else:
         G = synth.features(sg.n, F, 101, dev)
         dH = torch.empty_like(H)
+    if bf16:      # gathered matrices in bf16; the fp32 outputs keep their buffers
+        H = H.to(torch.bfloat16)
+        G = H if two_buffers else G.to(torch.bfloat16)
+        torch.cuda.empty_cache()
+    agg_fwd = g.dg_aggregate_fwd_bf16 if bf16 else g.dg_aggregate_fwd
+    agg_bwd = g.dg_aggregate_bwd_bf16 if bf16 else g.dg_aggregate_bwd
 
     # ---------------------------------------------------------------- device-resident timing
     def step():
-        g.dg_aggregate_fwd(H, op_code, out=out)
-        g.dg_aggregate_bwd(G, op_code, dH=dH)
+        agg_fwd(H, op_code, out=out)
+        agg_bwd(G, op_code, dH=dH)
 
     for _ in range(max(3, args.warmup)):
         step()
@@ -313,9 +323,9 @@ def main():
         torch.cuda.synchronize()
         marks[0].record(stream)
         for i in range(args.steps):
-            g.dg_aggregate_fwd(H, op_code, out=out)
+            agg_fwd(H, op_code, out=out)
             marks[2 * i + 1].record(stream)
-            g.dg_aggregate_bwd(G, op_code, dH=dH)
+            agg_bwd(G, op_code, dH=dH)
             marks[2 * i + 2].record(stream)
         torch.cuda.synchronize()
         if world > 1:
@@ -350,8 +360,9 @@ def main():
 
     # ---------------------------------------------------------------- roofline of the dominant kernel
     peak, peak_kind = measured_peaks()
-    b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False)
-    b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_rows_nonempty, op == "mean")
+    b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False, 2 if bf16 else 4)
+    b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_rows_nonempty, op == "mean",
+                             2 if bf16 else 4)
     dom = "fwd" if fwd_ms >= bwd_ms else "bwd"
     dom_ms, dom_bytes = (fwd_ms, b_fwd) if dom == "fwd" else (bwd_ms, b_bwd)
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9
@@ -359,7 +370,7 @@ def main():
     # handles that share of the edges and of the gathered matrix)
     per_call = max(1, round(launches / (2 * args.steps)))
     traffic = None
-    t = NCU_TRAFFIC.get((args.workload, F, op, args.scale))
+    t = None if bf16 else NCU_TRAFFIC.get((args.workload, F, op, args.scale))
     if t and t["version"] == binding.dg_version() and not args.set:
         traffic = t[dom] / per_call
     roofline = {
@@ -376,14 +387,15 @@ def main():
                 "edge_feat_per_s": sg.nnz * F / (fwd_ms * 1e-3)},
         "bwd": {"ms": bwd_ms, "bytes": b_bwd, "GBs": b_bwd / bwd_ms / 1e6,
                 "edge_feat_per_s": sg.nnz * F / (bwd_ms * 1e-3)},
-        "gather_bytes_per_launch": sg.nnz * F * 4,
-        "gather_GBs": sg.nnz * F * 4 / (dom_ms * 1e-3) / 1e9,
+        "gather_bytes_per_launch": sg.nnz * F * (2 if bf16 else 4),
+        "gather_GBs": sg.nnz * F * (2 if bf16 else 4) / (dom_ms * 1e-3) / 1e9,
     }
 
     # ---------------------------------------------------------------- GraphSAGE epoch (composite)
     epoch_info = None
     epoch_dims = {"reddit_like": [602, 256, 41], "products_like": [100, 256, 256, 47]}
-    if args.epochs > 0 and args.workload in epoch_dims and not args.feat and not two_buffers:
+    if (args.epochs > 0 and args.workload in epoch_dims and not args.feat and not two_buffers
+            and not bf16):
         from paper_2104_06700_b200 import graphsage
         dims = epoch_dims[args.workload]
         frac = 0.65 if args.workload == "reddit_like" else 196615 / 2449029
@@ -415,7 +427,7 @@ def main():
     if two_buffers:
         e2e = {"value": None, "unit": UNIT, "skipped": "host copies of the feature matrices of "
                "this workload exceed what the run pins; measured on the default workload"}
-    elif args.e2e_steps > 0:
+    elif args.e2e_steps > 0 and not bf16:
         Hh = torch.empty((sg.n, F), dtype=torch.float32).pin_memory()
         Gh = torch.empty((sg.n, F), dtype=torch.float32).pin_memory()
         Hh.copy_(H); Gh.copy_(G)
@@ -442,7 +454,7 @@ def main():
 
     # ---------------------------------------------------------------- CPU baseline (rank 0, N=1)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not two_buffers:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not two_buffers and not bf16:
         import oracle
         colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
         host = (sg.rowptr.cpu().numpy(), sg.colidx.cpu().numpy(),
@@ -465,7 +477,8 @@ def main():
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32" if not bf16 else "f32 sums over bf16-stored inputs", "data": "synthetic",
             "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
                        "F": F, "op": op, "weighted": weighted, "step": "fwd AP + bwd AP",
                        "replicas": world, "sorted_ids": bool(args.sorted_ids),
