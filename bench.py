@@ -415,7 +415,26 @@ def main():
         torch.cuda.synchronize()
         ep_ms = a.elapsed_time(b) / args.epochs
         calls = graphsage.aggregation_calls(dims)
+        # the algebraically equal order for layers that narrow: Linear first, then aggregate
+        torch.manual_seed(1234)
+        model_pf = graphsage.GraphSAGE(g, dims, project_first=True).to(dev)
+        run_pf = graphsage.make_epoch(model_pf, H, labels, train_idx)
+        for _ in range(3):
+            run_pf()
+        torch.cuda.synchronize()
+        a2, b2 = ev(), ev()
+        a2.record(stream)
+        for _ in range(args.epochs):
+            run_pf()
+        b2.record(stream)
+        torch.cuda.synchronize()
+        pf_calls = graphsage.aggregation_calls(dims, True)
+        del model_pf, run_pf
         epoch_info = {"ms_per_epoch": ep_ms, "epochs": args.epochs, "dims": dims,
+                      "project_first": {"ms_per_epoch": a2.elapsed_time(b2) / args.epochs,
+                                        "aggregations": [f"{d}:{w}" for d, w in pf_calls],
+                                        "note": "Linear before the aggregation where a layer "
+                                                "narrows; same function up to fp32 rounding"},
                       "train_vertices": int(train_idx.numel()), "loss": float(last_loss),
                       "aggregations": [f"{d}:{w}" for d, w in calls],
                       "ap_edge_feat_per_epoch": sg.nnz * sum(w for _, w in calls),

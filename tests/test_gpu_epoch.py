@@ -25,13 +25,14 @@ def reference_forward(sg, X, weights, biases):
     return H
 
 
+@pytest.mark.parametrize("project_first", [False, True])
 @pytest.mark.parametrize("dims", [[64, 32, 7], [20, 16, 16, 5]])
-def test_epoch_loss_and_gradients_match_torch_reference(dims):
+def test_epoch_loss_and_gradients_match_torch_reference(dims, project_first):
     sg = synth.make("tiny", weighted=False)
     g = make_graph(sg)
     g.dg_graph_transpose()
     torch.manual_seed(0)
-    model = graphsage.GraphSAGE(g, dims).to(DEV)
+    model = graphsage.GraphSAGE(g, dims, project_first=project_first).to(DEV)
     X = synth.features(sg.n, dims[0], 3, DEV)
     labels = torch.randint(0, dims[-1], (sg.n,), device=DEV)
     train_idx = torch.arange(0, sg.n, 3, device=DEV)
@@ -65,3 +66,7 @@ def test_epoch_function_trains():
     losses = [float(epoch()) for _ in range(30)]
     assert losses[-1] < losses[0]
     assert graphsage.aggregation_calls([64, 32, 7]) == [("fwd", 64), ("fwd", 32), ("bwd", 32)]
+    assert graphsage.aggregation_calls([64, 32, 7], True) == [("fwd", 32), ("bwd", 32),
+                                                              ("fwd", 7), ("bwd", 7)]
+    assert graphsage.aggregation_calls([16, 32, 32, 7], True) == [
+        ("fwd", 16), ("fwd", 32), ("bwd", 32), ("fwd", 7), ("bwd", 7)]
