@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 
 METRIC = "ap_fwd_bwd_edge_feat_per_s"
 UNIT = "edge*feat/s"
-NORTH_STAR_HBM_GBS = 8000.0
+NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one dg_aggregate_fwd / _bwd call,
 # summed over its launches, from the ncu captures summarised under profiles/.  Reported as
 # roofline.traffic only while the library still has the version the capture was taken with.
@@ -378,7 +378,7 @@ def main():
         "kernel": ("ap_kernel_r48" if (weighted or (dom == "bwd" and op == "mean")) and F >= 64
                    else "ap_kernel") + f" ({dom}: {per_call} launch(es) per dg_aggregate_{dom} call)",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "peak_kind": f"of {peak_kind}", "frac_of_north_star_8TBs": achieved / NORTH_STAR_HBM_GBS,
+        "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "launches_per_call": per_call,
         "algorithmic_bytes_per_launch": dom_bytes / per_call, "ms_per_launch": dom_ms / per_call,
         "traffic": traffic,
