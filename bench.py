@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"],
                     help="storage of the gathered matrices (sums and outputs are fp32 either "
                          "way); bf16 is reported separately, the headline is f32")
+    ap.add_argument("--probe", action="store_true",
+                    help="measure the gather ceilings of this GPU (dg_probe_gather) and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sorted-ids", action="store_true",
                     help="keep the generator's construction order of vertex ids (communities "
@@ -224,10 +226,46 @@ def run_reference(args):
     }))
 
 
+def run_probe():
+    """Random-row gather rates from an L2-resident and from an HBM-sized table (one JSON line)."""
+    import torch
+    from paper_2104_06700_b200 import binding
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    stream = torch.cuda.current_stream()
+    count = 1 << 26
+    sink = torch.empty(((count + 511) // 512) * 128, dtype=torch.float32, device=dev)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    out = {"probe": "dg_probe_gather", "gathers": count, "unit": "GB/s of gathered bytes"}
+    for label, table_bytes in (("l2_30MB", 30e6), ("hbm_16GB", 16e9)):
+        for row_floats in (128, 64, 32):
+            rows = int(table_bytes // (row_floats * 4))
+            table = torch.zeros((rows, row_floats), dtype=torch.float32, device=dev)
+            idx = torch.randint(0, rows, (count,), generator=gen, device=dev, dtype=torch.int32)
+            for _ in range(3):
+                binding.dg_probe_gather(table, idx, sink)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(5):
+                binding.dg_probe_gather(table, idx, sink)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / 5
+            out[f"{label}_row{row_floats * 4}B"] = count * row_floats * 4 / (ms * 1e-3) / 1e9
+            del table, idx
+            torch.cuda.empty_cache()
+    print(json.dumps(out))
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+        return
+    if args.probe:
+        run_probe()
         return
 
     import torch

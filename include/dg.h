@@ -207,6 +207,20 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
 dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);
 dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value);
 
+/*
+ * Diagnostic: gathers `count` rows table[idx[i]] (rows of row_floats fp32, a power of two in
+ * [4, 128]; idx values in [0, rows)) and sums them per warp, 512 gathers per warp, with the
+ * load pattern of the aggregation kernels and nothing else.  Timed by the caller, it gives the
+ * rate at which this GPU delivers gathered rows from L2 (small table) or from HBM (table far
+ * larger than L2): the ceilings the aggregation rates are compared with.
+ *   table  device, rows x row_floats fp32, 16-byte aligned
+ *   idx    device, count int32
+ *   sink   device, 16-byte aligned, >= ceil(count / 512) * 128 floats; receives the warp sums
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_probe_gather(const float* table, int64_t rows, int32_t row_floats,
+                            const int32_t* idx, int64_t count, float* sink, void* stream);
+
 /* Number of kernels the library has launched from this process (all handles, all threads). */
 int64_t dg_kernel_launch_count(void);
 

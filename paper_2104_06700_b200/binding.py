@@ -28,7 +28,7 @@ EXPORTS = [
     "dg_graph_transpose", "dg_graph_transpose_static", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
     "dg_aggregate_fwd_bf16", "dg_aggregate_bwd_bf16",
     "dg_aggregate_host_workspace", "dg_aggregate_host", "dg_graph_set_param",
-    "dg_graph_get_param", "dg_kernel_launch_count", "dg_last_error", "dg_version",
+    "dg_graph_get_param", "dg_probe_gather", "dg_kernel_launch_count", "dg_last_error", "dg_version",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -69,6 +69,7 @@ def lib() -> ctypes.CDLL:
         L.dg_aggregate_host.argtypes = [p, p, p, i32, ctypes.c_int, p, p, p, sz, p]
         L.dg_graph_set_param.argtypes = [p, ctypes.c_char_p, i64]
         L.dg_graph_get_param.argtypes = [p, ctypes.c_char_p, ctypes.POINTER(i64)]
+        L.dg_probe_gather.argtypes = [p, i64, i32, p, i64, p, p]
         L.dg_kernel_launch_count.restype = i64
         L.dg_last_error.restype = ctypes.c_char_p
         L.dg_version.restype = ctypes.c_char_p
@@ -112,6 +113,13 @@ def dg_last_error() -> str:
 
 def dg_kernel_launch_count() -> int:
     return int(lib().dg_kernel_launch_count())
+
+
+def dg_probe_gather(table: torch.Tensor, idx: torch.Tensor, sink: torch.Tensor, stream=None) -> None:
+    """Wraps ``dg_probe_gather``: table (rows, row_floats) fp32, idx int32, sink fp32."""
+    _check(lib().dg_probe_gather(_dev_ptr(table, torch.float32, "table"), table.shape[0],
+                                 table.shape[1], _dev_ptr(idx, torch.int32, "idx"), idx.numel(),
+                                 _dev_ptr(sink, torch.float32, "sink"), _stream(stream)))
 
 
 def dg_graph_create(n: int, nnz: int, rowptr: torch.Tensor, colidx: torch.Tensor,

@@ -259,6 +259,20 @@ def test_feature_width_limit_and_parameter_ranges(tiny):
         g.dg_graph_get_param(name)
 
 
+def test_probe_gather_sums_the_rows_it_names():
+    rows, rf, count = 1000, 32, 5000
+    table = synth.features(rows, rf, 1, DEV)
+    idx = torch.randint(0, rows, (count,), device=DEV, dtype=torch.int32)
+    sink = torch.zeros(((count + 511) // 512) * 128, device=DEV)
+    binding.dg_probe_gather(table, idx, sink)
+    torch.cuda.synchronize()
+    # warp w sums gathers [512 w, 512 w + 512): 32 lanes x 4 floats hold 4 lane groups x 32 columns
+    got = sink.view(-1, 4, rf).sum(1)
+    want = torch.stack([table[idx[w * 512:(w + 1) * 512].long()].double().sum(0)
+                        for w in range(got.shape[0])])
+    assert torch.allclose(got.double(), want, rtol=1e-4, atol=1e-3)
+
+
 # ------------------------------------------------------------------ errors never trap
 def test_error_statuses(tiny):
     g = make_graph(tiny)
