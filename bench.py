@@ -61,6 +61,8 @@ def parse_args():
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"],
                     help="storage of the gathered matrices (sums and outputs are fp32 either "
                          "way); bf16 is reported separately, the headline is f32")
+    ap.add_argument("--no-probe", action="store_true",
+                    help="skip the two gather-ceiling measurements added to the roofline object")
     ap.add_argument("--probe", action="store_true",
                     help="measure the gather ceilings of this GPU (dg_probe_gather) and exit")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -224,6 +226,27 @@ def run_reference(args):
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def probe_rate(binding, torch, dev, table_bytes, row_floats, count=1 << 25, reps=3):
+    """GB/s of gathered bytes dg_probe_gather reaches on a table of the given size."""
+    rows = int(table_bytes // (row_floats * 4))
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(0)
+    table = torch.zeros((rows, row_floats), dtype=torch.float32, device=dev)
+    idx = torch.randint(0, rows, (count,), generator=gen, device=dev, dtype=torch.int32)
+    sink = torch.empty(((count + 511) // 512) * 128, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(2):
+        binding.dg_probe_gather(table, idx, sink)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(stream)
+    for _ in range(reps):
+        binding.dg_probe_gather(table, idx, sink)
+    b.record(stream)
+    torch.cuda.synchronize()
+    return count * row_floats * 4 / (a.elapsed_time(b) / reps * 1e-3) / 1e9
 
 
 def run_probe():
@@ -428,6 +451,16 @@ def main():
         "gather_bytes_per_launch": sg.nnz * F * (2 if bf16 else 4),
         "gather_GBs": sg.nnz * F * (2 if bf16 else 4) / (dom_ms * 1e-3) / 1e9,
     }
+
+    # what this GPU can deliver to a gather at all: the aggregation's own ceilings
+    if rank == 0 and world == 1 and not args.no_probe and not two_buffers:
+        l2_c = probe_rate(binding, torch, dev, 30e6, 128)
+        hbm_c = probe_rate(binding, torch, dev, 8e9, 128)
+        roofline["gather_ceilings"] = {
+            "how": "dg_probe_gather, random 512-byte rows, 30 MB table (L2) and 8 GB table (HBM)",
+            "l2_GBs": l2_c, "hbm_GBs": hbm_c,
+            "gathered_frac_of_l2_ceiling": roofline["gather_GBs"] / l2_c,
+            "gathered_frac_of_hbm_ceiling": roofline["gather_GBs"] / hbm_c}
 
     # ---------------------------------------------------------------- GraphSAGE epoch (composite)
     epoch_info = None
