@@ -8,7 +8,15 @@ training, where the graph is static over epochs); they are timed separately and 
 "ingest".  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                  [--workload NAME] [--scale S] [--feat F] [--op sum|mean]
+                  [--workload NAME] [--scale S] [--feat F] [--op sum|mean] [--dtype f32|bf16]
+                  [--set knob=value ...] [--sorted-ids] [--epochs E] [--e2e-steps S]
+                  [--no-cpu-baseline] [--no-probe]
+  python bench.py --probe        # only the gather ceilings of this GPU
+
+Beside the device-resident step the line carries: the roofline object of the slower of the two
+calls (compulsory bytes, DRAM traffic from the ncu captures, gather ceilings measured in the
+same run), the same step end to end from pinned host memory ("e2e"), the CPU oracle on a row
+sample ("cpu_baseline"), and the time of one full-batch GraphSAGE epoch ("epoch").
 
 N > 1 (under torchrun): the path has no exchange step and is not sharded, so every rank runs
 an independent replica of the same workload; the value is the units all ranks processed over
