@@ -99,3 +99,33 @@ def test_random_dense_graph_with_source_blocks(seed):
         H = synth.features(n, F, 17 + seed, DEV)
         G = synth.features(n, F, 18 + seed, DEV)
         check_fwd_bwd(g, (rowptr, col, w), H, G, int(rng.integers(0, 2)), csc)
+
+
+def test_extreme_shapes():
+    """One vertex with thousands of self-loops; a handful of vertices with the widest feature
+    rows the library accepts (2^20 columns: 2048 feature slices in one launch)."""
+    rng = np.random.default_rng(77)
+    n, nnz = 1, 5000
+    rowptr = np.array([0, nnz], dtype=np.int64)
+    col = np.zeros(nnz, dtype=np.int32)
+    w = rng.random(nnz).astype(np.float32)
+    g = binding.dg_graph_create(n, nnz, torch.as_tensor(rowptr, device=DEV),
+                                torch.as_tensor(col, device=DEV), torch.as_tensor(w, device=DEV))
+    csc = check_transpose(g, rowptr, col, w)
+    H, G = synth.features(n, 40, 1, DEV), synth.features(n, 40, 2, DEV)
+    for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+        check_fwd_bwd(g, (rowptr, col, w), H, G, op, csc)
+
+    n, F = 5, 1 << 20
+    rows = [[1, 2], [0], [], [0, 1, 2, 3, 4], [4]]
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    rowptr[1:] = np.cumsum([len(r) for r in rows])
+    col = np.concatenate([np.asarray(r, dtype=np.int32) for r in rows])
+    g = binding.dg_graph_create(n, len(col), torch.as_tensor(rowptr, device=DEV),
+                                torch.as_tensor(col, device=DEV), None)
+    csc = check_transpose(g, rowptr, col, None)
+    H, G = synth.features(n, F, 3, DEV), synth.features(n, F, 4, DEV)
+    check_fwd_bwd(g, (rowptr, col, None), H, G, binding.DG_OP_MEAN, csc)
+    out = g.dg_aggregate_fwd_bf16(H.to(torch.bfloat16), binding.DG_OP_SUM)
+    assert torch.allclose(out, g.dg_aggregate_fwd(H.to(torch.bfloat16).float(), binding.DG_OP_SUM),
+                          rtol=1e-4, atol=1e-4)
