@@ -509,13 +509,14 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
   ap_body<E, VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
 
-// The same kernel compiled for five resident blocks per SM (at most 48 registers).  The scaled
-// variants with up to four floats per lane and step (and at least 16 lanes per edge) carry the edge factors on top of everything
-// else and would take 60 registers; measured on B200 the higher occupancy wins for them
-// (Reddit-like backward 22.0 -> 19.3 ms, Products-like backward 7.0 -> 6.2 ms), while the same
-// cap slows the unscaled variants down.
+// The same kernel compiled for six resident blocks per SM (at most 40 registers).  The scaled
+// variants with up to 16 bytes per lane and step (and at least 16 lanes per edge) carry the
+// edge factors on top of everything else and would take 60 registers; measured on B200 the
+// higher occupancy wins for them (Reddit-like backward 22.0 ms uncapped, 19.2 ms at five
+// blocks, 18.3 ms at six, 20.0 ms at seven or eight; Products-like backward 7.0 -> 5.9 ms),
+// while a cap slows the unscaled variants down.
 template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
-__global__ void __launch_bounds__(kBlock, 5) ap_kernel_r48(const ApArgs a, const int heavy_blocks) {
+__global__ void __launch_bounds__(kBlock, 6) ap_kernel_r40(const ApArgs a, const int heavy_blocks) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
   ap_body<E, VEC, G, CPL, SCALED, SEG>(a, heavy_blocks, part);
 }
@@ -537,8 +538,8 @@ dg_status_t launch_pair(const Graph* g, const ApArgs& a, int slices, cudaStream_
   if (a.n == 0) return DG_OK;
   void (*kernel)(const ApArgs, const int);
   if constexpr (SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16) {
-    kernel = a.seg_lo ? ap_kernel_r48<E, VEC, G, CPL, SCALED, true>
-                      : ap_kernel_r48<E, VEC, G, CPL, SCALED, false>;
+    kernel = a.seg_lo ? ap_kernel_r40<E, VEC, G, CPL, SCALED, true>
+                      : ap_kernel_r40<E, VEC, G, CPL, SCALED, false>;
   } else {
     kernel = a.seg_lo ? ap_kernel<E, VEC, G, CPL, SCALED, true>
                       : ap_kernel<E, VEC, G, CPL, SCALED, false>;
