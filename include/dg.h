@@ -193,7 +193,10 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *   "heavy_threshold"  rows longer than this are summed by a whole thread block
  *   "heavy_blocks_per_sm"  thread blocks per SM that walk the list of heavy rows (longest first)
  *                      before the launch turns to the light rows; 0 = as many as are resident
- *   "slice_features"   features per pass over the graph (0 = choose from the L2 size)
+ *   "slice_features"   features per pass over the graph (0 = choose from the L2 size; a value
+ *                      that would need more than 65535 passes is widened)
+ * Changing "heavy_threshold" rebuilds the heavy lists on the default stream and waits for it:
+ * do not change it while aggregations of this handle are in flight.
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
  *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows;
  *                      0 = about 1024 edges per warp, between 32 and 248 rows per block)

@@ -650,6 +650,10 @@ dg_status_t aggregate_run(const Graph* g, const ApArgs& a0, const int32_t* split
   }
   slice = (slice / vec) * vec;
   if (slice < vec) slice = vec;
+  if ((a.F + slice - 1) / slice > 65535) {  // grid.y limit: widen a (requested) tiny slice
+    slice = (a.F + 65534) / 65535;
+    slice = ((slice + vec - 1) / vec) * vec;
+  }
   // even out the slices: same count, smallest width that covers F
   const int64_t nsl = (a.F + slice - 1) / slice;
   int64_t even = (a.F + nsl - 1) / nsl;

@@ -126,6 +126,9 @@ def test_extreme_shapes():
     csc = check_transpose(g, rowptr, col, None)
     H, G = synth.features(n, F, 3, DEV), synth.features(n, F, 4, DEV)
     check_fwd_bwd(g, (rowptr, col, None), H, G, binding.DG_OP_MEAN, csc)
+    g.dg_graph_set_param("slice_features", 1)      # would be 2^20 slices: the library widens it
+    check_fwd_bwd(g, (rowptr, col, None), H, G, binding.DG_OP_SUM, csc)
+    g.dg_graph_set_param("slice_features", 0)
     out = g.dg_aggregate_fwd_bf16(H.to(torch.bfloat16), binding.DG_OP_SUM)
     assert torch.allclose(out, g.dg_aggregate_fwd(H.to(torch.bfloat16).float(), binding.DG_OP_SUM),
                           rtol=1e-4, atol=1e-4)
