@@ -195,8 +195,6 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *                      before the launch turns to the light rows; 0 = as many as are resident
  *   "slice_features"   features per pass over the graph (0 = choose from the L2 size; a value
  *                      that would need more than 65535 passes is widened)
- * Changing "heavy_threshold" rebuilds the heavy lists on the default stream and waits for it:
- * do not change it while aggregations of this handle are in flight.
  *   "rows_per_block"   destination rows per thread block in the light-row kernel (1..248,
  *                      rounded up to a multiple of 8: each of the 8 warps owns a run of rows;
  *                      0 = about 1024 edges per warp, between 32 and 248 rows per block)
@@ -205,6 +203,8 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,
  *                      4, 8 or 16; ignored for graphs without split pointers, i.e. with fewer
  *                      than 64 edges per vertex or unsorted rows)
+ * Changing "heavy_threshold" rebuilds the heavy lists on the default stream and waits for it:
+ * do not change it while aggregations of this handle are in flight.
  * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.
  */
 dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);
