@@ -178,7 +178,7 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (e != cudaSuccess) { delete g; return cuda_fail(e, "cudaGetDeviceProperties"); }
   g->sm_count = prop.multiProcessorCount;
   g->l2_bytes = (size_t)prop.l2CacheSize;
-  g->l2_budget_bytes = (int64_t)(g->l2_bytes * 3 / 10);
+  g->l2_budget_bytes = (int64_t)(g->l2_bytes * 19 / 40);  // 60 of 126 MB measured best on B200
   g->fine_rows = (n + kFineBlocks - 1) / kFineBlocks;
   if (g->fine_rows < 1) g->fine_rows = 1;
   g->heavy_cap = nnz / 64 + 1;  // enough for any threshold >= 64
