@@ -509,11 +509,27 @@ def main():
         torch.cuda.synchronize()
         pf_calls = graphsage.aggregation_calls(dims, True)
         del model_pf, run_pf
+        # the same, aggregating bf16-rounded activations (mixed precision; not the headline)
+        torch.manual_seed(1234)
+        model_bf = graphsage.GraphSAGE(g, dims, project_first=True, bf16_aggregate=True).to(dev)
+        run_bf = graphsage.make_epoch(model_bf, H, labels, train_idx)
+        for _ in range(3):
+            run_bf()
+        torch.cuda.synchronize()
+        a3, b3 = ev(), ev()
+        a3.record(stream)
+        for _ in range(args.epochs):
+            run_bf()
+        b3.record(stream)
+        torch.cuda.synchronize()
+        del model_bf, run_bf
         epoch_info = {"ms_per_epoch": ep_ms, "epochs": args.epochs, "dims": dims,
                       "project_first": {"ms_per_epoch": a2.elapsed_time(b2) / args.epochs,
                                         "aggregations": [f"{d}:{w}" for d, w in pf_calls],
                                         "note": "Linear before the aggregation where a layer "
-                                                "narrows; same function up to fp32 rounding"},
+                                                "narrows; same function up to fp32 rounding",
+                                        "ms_per_epoch_bf16_aggregation":
+                                            a3.elapsed_time(b3) / args.epochs},
                       "train_vertices": int(train_idx.numel()), "loss": float(last_loss),
                       "aggregations": [f"{d}:{w}" for d, w in calls],
                       "ap_edge_feat_per_epoch": sg.nnz * sum(w for _, w in calls),

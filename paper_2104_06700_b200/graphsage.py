@@ -18,24 +18,32 @@ from . import binding
 
 
 class _Aggregate(torch.autograd.Function):
-    """out = A H through dg_aggregate_fwd; the backward pass calls dg_aggregate_bwd."""
+    """out = A H through dg_aggregate_fwd; the backward pass calls dg_aggregate_bwd.  With
+    ``bf16`` the gathered matrices (H in the forward, dOut in the backward pass) are rounded to
+    bf16 first and the bf16 entry points are used; sums and results stay fp32."""
 
     @staticmethod
-    def forward(ctx, H: torch.Tensor, graph: "binding.Graph", op: int) -> torch.Tensor:
-        ctx.graph, ctx.op = graph, op
+    def forward(ctx, H: torch.Tensor, graph: "binding.Graph", op: int, bf16: bool) -> torch.Tensor:
+        ctx.graph, ctx.op, ctx.bf16 = graph, op, bf16
+        if bf16:
+            return graph.dg_aggregate_fwd_bf16(H.contiguous().to(torch.bfloat16), op)
         return graph.dg_aggregate_fwd(H.contiguous(), op)
 
     @staticmethod
     def backward(ctx, dOut: torch.Tensor):
         dH = None
         if ctx.needs_input_grad[0]:
-            dH = ctx.graph.dg_aggregate_bwd(dOut.contiguous(), ctx.op)
-        return dH, None, None
+            if ctx.bf16:
+                dH = ctx.graph.dg_aggregate_bwd_bf16(dOut.contiguous().to(torch.bfloat16), ctx.op)
+            else:
+                dH = ctx.graph.dg_aggregate_bwd(dOut.contiguous(), ctx.op)
+        return dH, None, None, None
 
 
-def aggregate(graph: "binding.Graph", H: torch.Tensor, op: int = binding.DG_OP_SUM) -> torch.Tensor:
+def aggregate(graph: "binding.Graph", H: torch.Tensor, op: int = binding.DG_OP_SUM,
+              bf16: bool = False) -> torch.Tensor:
     """Differentiable aggregation primitive (the graph must have been transposed)."""
-    return _Aggregate.apply(H, graph, op)
+    return _Aggregate.apply(H, graph, op, bf16)
 
 
 class GraphSAGE(torch.nn.Module):
@@ -48,10 +56,12 @@ class GraphSAGE(torch.nn.Module):
     aggregates first (its Table 8 counts the aggregation at the layers' input widths).
     """
 
-    def __init__(self, graph: "binding.Graph", dims: Sequence[int], project_first: bool = False):
+    def __init__(self, graph: "binding.Graph", dims: Sequence[int], project_first: bool = False,
+                 bf16_aggregate: bool = False):
         super().__init__()
         self.graph = graph
         self.project_first = project_first
+        self.bf16_aggregate = bf16_aggregate   # aggregate bf16-rounded activations (even widths)
         self.lin = torch.nn.ModuleList(
             [torch.nn.Linear(dims[i], dims[i + 1]) for i in range(len(dims) - 1)])
         deg = (graph.rowptr[1:] - graph.rowptr[:-1]).to(torch.float32)
@@ -61,9 +71,11 @@ class GraphSAGE(torch.nn.Module):
         for i, lin in enumerate(self.lin):
             if self.project_first and lin.out_features < lin.in_features:
                 P = torch.nn.functional.linear(H, lin.weight)           # bias after the mean
-                H = (aggregate(self.graph, P, binding.DG_OP_SUM) + P) * self.inv_deg1 + lin.bias
+                bf = self.bf16_aggregate and P.shape[1] % 2 == 0
+                H = (aggregate(self.graph, P, binding.DG_OP_SUM, bf) + P) * self.inv_deg1 + lin.bias
             else:
-                Z = (aggregate(self.graph, H, binding.DG_OP_SUM) + H) * self.inv_deg1
+                bf = self.bf16_aggregate and H.shape[1] % 2 == 0
+                Z = (aggregate(self.graph, H, binding.DG_OP_SUM, bf) + H) * self.inv_deg1
                 H = lin(Z)
             if i + 1 < len(self.lin):
                 H = torch.relu(H)

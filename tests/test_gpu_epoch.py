@@ -70,3 +70,23 @@ def test_epoch_function_trains():
                                                               ("fwd", 7), ("bwd", 7)]
     assert graphsage.aggregation_calls([16, 32, 32, 7], True) == [
         ("fwd", 16), ("fwd", 32), ("bwd", 32), ("fwd", 7), ("bwd", 7)]
+
+
+def test_bf16_aggregation_stays_close_to_fp32():
+    """Aggregating bf16-rounded activations changes the loss by bf16 rounding only."""
+    sg = synth.make("tiny", weighted=False)
+    g = make_graph(sg)
+    g.dg_graph_transpose()
+    X = synth.features(sg.n, 64, 3, DEV)
+    labels = torch.randint(0, 8, (sg.n,), device=DEV)
+    losses = []
+    for bf in (False, True):
+        torch.manual_seed(0)
+        model = graphsage.GraphSAGE(g, [64, 32, 8], bf16_aggregate=bf).to(DEV)
+        logits = model(X)
+        loss = torch.nn.functional.cross_entropy(logits, labels)
+        loss.backward()
+        losses.append((float(loss), model.lin[0].weight.grad.clone()))
+    assert abs(losses[0][0] - losses[1][0]) <= 2e-2 * abs(losses[0][0])
+    scale = float(losses[0][1].abs().max())
+    assert float((losses[0][1] - losses[1][1]).abs().max()) <= 5e-2 * scale
