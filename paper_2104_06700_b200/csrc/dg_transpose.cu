@@ -8,9 +8,9 @@
 //   1. digit_histogram : per tile of kTile keys, the number of keys per digit -> hist[digit][tile]
 //   2. exclusive scan of hist (digit-major, so the scan yields global output offsets):
 //      scan_reduce -> scan_spine (one block) -> scan_apply
-//   3. digit_scatter   : ranks every key inside its tile in input order (match.any inside a warp,
-//      per-warp counters across rounds, a fixed pass across the warps), stages the tile sorted by
-//      digit in shared memory and writes each digit run to its global offset.
+//   3. digit_scatter   : ranks every key inside its tile in input order (ballots over the digit
+//      bits inside a warp, per-warp counters across rounds, a fixed pass across the warps), stages
+//      the tile sorted by digit in shared memory and writes each digit run to its global offset.
 // Stability of every step makes the final order (key, k) ascending.  After the last pass the
 // sorted keys give colptr by boundary detection, and perm gives rowidx_T and w_T by gathers.
 #include "dg_internal.cuh"
@@ -33,17 +33,35 @@ __device__ __forceinline__ uint32_t digit_of(uint32_t key, int shift) {
   return (key >> shift) & (kRadix - 1);
 }
 
+// A thread reads its keys as 16-byte vectors when the array allows it (four loads in flight
+// then cover the whole tile; with 4-byte loads the kernel waited on memory at a third of the
+// copy bandwidth).  The caller's colidx, the keys of the first pass, is only 4-byte aligned in
+// general: `vector_ok` says whether keys is 16-byte aligned.
 __global__ void __launch_bounds__(kSortBlock)
 digit_histogram(const uint32_t* __restrict__ keys, int64_t count, int shift, int64_t tiles,
-                uint32_t* __restrict__ hist) {
+                int vector_ok, uint32_t* __restrict__ hist) {
   __shared__ uint32_t h[kRadix];
   h[threadIdx.x] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kTile;
+  if (vector_ok && base + kTile <= count) {
+    const uint4* v = reinterpret_cast<const uint4*>(keys + base);
+    uint4 k[kItems / 4];
+#pragma unroll
+    for (int i = 0; i < kItems / 4; ++i) k[i] = v[i * kSortBlock + threadIdx.x];
+#pragma unroll
+    for (int i = 0; i < kItems / 4; ++i) {
+      atomicAdd(&h[digit_of(k[i].x, shift)], 1u);
+      atomicAdd(&h[digit_of(k[i].y, shift)], 1u);
+      atomicAdd(&h[digit_of(k[i].z, shift)], 1u);
+      atomicAdd(&h[digit_of(k[i].w, shift)], 1u);
+    }
+  } else {
 #pragma unroll 4
-  for (int i = 0; i < kItems; ++i) {
-    const int64_t k = base + i * kSortBlock + threadIdx.x;
-    if (k < count) atomicAdd(&h[digit_of(keys[k], shift)], 1u);
+    for (int i = 0; i < kItems; ++i) {
+      const int64_t k = base + i * kSortBlock + threadIdx.x;
+      if (k < count) atomicAdd(&h[digit_of(keys[k], shift)], 1u);
+    }
   }
   __syncthreads();
   hist[(int64_t)threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];
@@ -124,14 +142,36 @@ scan_apply(uint32_t* __restrict__ data, int64_t m, const uint32_t* __restrict__ 
   }
 }
 
+// Lanes of the warp that hold the same digit as this lane (lanes without a key only match one
+// another): one ballot per digit bit, each keeping the lanes that agree with this lane on that
+// bit.  Unlike match.any, whose cost grows with the number of distinct values in the warp (about
+// 30 for the random low digits of vertex ids), this costs the same for every digit mix.
+__device__ __forceinline__ unsigned digit_peers(uint32_t d, bool valid) {
+  const unsigned have = __ballot_sync(kFull, valid);
+  unsigned peers = valid ? have : ~have;
+#pragma unroll
+  for (int b = 0; b < kRadixBits; ++b) {
+    const bool bit = (d >> b) & 1u;
+    const unsigned m = __ballot_sync(kFull, bit);
+    peers &= bit ? m : ~m;
+  }
+  return peers;
+}
+
 // ---- stable scatter of one tile ----
 // vals_in == nullptr means "the value of key k is k" (first pass).  keys_out may be nullptr when
 // the sorted keys are not needed (never the case for the last pass, which feeds colptr).
-__global__ void __launch_bounds__(kSortBlock)
+// Four blocks per SM (64 registers a thread): the ranking is a chain of shared-memory and
+// ballot latencies, and the fourth block hides more of it than the few spilled words cost
+// (three blocks at 80 registers were 10 % slower, five with the values read late 3 % slower).
+__global__ void __launch_bounds__(kSortBlock, 4)
 digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
               int64_t count, int shift, int64_t tiles, const uint32_t* __restrict__ offsets,
               uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out) {
-  __shared__ uint32_t warp_cnt[kSortWarps][kRadix];
+  // A warp ranks its 512 keys as two streams of 256 (rounds 0..7 and 8..15), each with its own
+  // counters, so that two independent chains of counter updates are in flight at a time.
+  __shared__ uint16_t cnt_a[kSortWarps][kRadix];
+  __shared__ uint16_t cnt_b[kSortWarps][kRadix];
   __shared__ uint32_t digit_base[kRadix];
   __shared__ uint32_t global_base[kRadix];
   __shared__ uint32_t skeys[kTile];
@@ -142,7 +182,12 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
   const int64_t remaining = count - tile_base;
   const int tile_count = remaining < kTile ? (int)remaining : kTile;
 
-  for (int w = 0; w < kSortWarps; ++w) warp_cnt[w][threadIdx.x] = 0;
+  // this tile's global offset of digit threadIdx.x: fetched now, needed after the ranking
+  const uint32_t my_global_base = offsets[(int64_t)threadIdx.x * tiles + blockIdx.x];
+  for (int w = 0; w < kSortWarps; ++w) {
+    cnt_a[w][threadIdx.x] = 0;
+    cnt_b[w][threadIdx.x] = 0;
+  }
   __syncthreads();
 
   // Warp `warp` owns keys [warp*512, warp*512+512) of the tile, 32 consecutive keys per round,
@@ -156,33 +201,46 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
     const bool valid = local < tile_count;
     key[r] = valid ? keys_in[tile_base + local] : 0u;
     val[r] = valid ? (vals_in ? vals_in[tile_base + local] : (uint32_t)(tile_base + local)) : 0u;
-    const uint32_t d = valid ? digit_of(key[r], shift) : (uint32_t)kRadix;  // kRadix = "none"
-    const unsigned peers = __match_any_sync(kFull, d);
-    const int leader = __ffs(peers) - 1;
-    uint32_t before = 0;
-    if (valid && lane == leader) {
-      before = warp_cnt[warp][d];
-      warp_cnt[warp][d] = before + __popc(peers);
+  }
+  constexpr int kHalf = kItems / 2;
+#pragma unroll
+  for (int r = 0; r < kHalf; ++r) {
+#pragma unroll
+    for (int stream = 0; stream < 2; ++stream) {
+      const int rr = r + stream * kHalf;
+      uint16_t* cnt = stream ? cnt_b[warp] : cnt_a[warp];
+      const bool valid = warp * (32 * kItems) + rr * 32 + lane < tile_count;
+      const uint32_t d = valid ? digit_of(key[rr], shift) : 0u;
+      const unsigned peers = digit_peers(d, valid);
+      const int leader = __ffs(peers) - 1;
+      uint32_t before = 0;
+      if (valid && lane == leader) {
+        before = cnt[d];
+        cnt[d] = (uint16_t)(before + __popc(peers));
+      }
+      before = __shfl_sync(kFull, before, leader);
+      rank[rr] = (uint16_t)(before + __popc(peers & lt_mask));
     }
-    before = __shfl_sync(kFull, before, leader);
-    rank[r] = (uint16_t)(before + __popc(peers & lt_mask));
     __syncwarp();
   }
   __syncthreads();
 
-  // thread t owns digit t: exclusive prefix over the warps, then over the digits
+  // thread t owns digit t: exclusive prefix over (warp, stream), then over the digits
   {
     const int d = threadIdx.x;
     uint32_t run = 0;
 #pragma unroll
     for (int w = 0; w < kSortWarps; ++w) {
-      const uint32_t c = warp_cnt[w][d];
-      warp_cnt[w][d] = run;
-      run += c;
+      const uint32_t ca = cnt_a[w][d];
+      cnt_a[w][d] = (uint16_t)run;
+      run += ca;
+      const uint32_t cb = cnt_b[w][d];
+      cnt_b[w][d] = (uint16_t)run;
+      run += cb;
     }
     uint32_t total;
     digit_base[d] = block_exclusive_scan(run, &total);
-    global_base[d] = offsets[(int64_t)d * tiles + blockIdx.x];
+    global_base[d] = my_global_base;
   }
   __syncthreads();
 
@@ -191,7 +249,8 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
     const int local = warp * (32 * kItems) + r * 32 + lane;
     if (local < tile_count) {
       const uint32_t d = digit_of(key[r], shift);
-      const uint32_t pos = digit_base[d] + warp_cnt[warp][d] + rank[r];
+      const uint32_t in_digit = r < kHalf ? cnt_a[warp][d] : cnt_b[warp][d];
+      const uint32_t pos = digit_base[d] + in_digit + rank[r];
       skeys[pos] = key[r];
       svals[pos] = val[r];
     }
@@ -207,16 +266,33 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
   }
 }
 
-// colptr[u] = first position q whose sorted key is >= u.  Thread q fills the ids between the
-// key before it and its own key; thread nnz closes the array up to n.
+// colptr[u] = first position q whose sorted key is >= u.  Position q fills the ids between the
+// key before it and its own key; position nnz closes the array up to n.  A thread takes
+// kColptrItems consecutive positions (one 16-byte load when `vector_ok`: sorted 16-byte aligned).
+constexpr int kColptrItems = 4;
 __global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int64_t nnz,
-                                        int64_t n, int64_t* __restrict__ colptr) {
-  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (q > nnz) return;
-  const int64_t prev = q > 0 ? (int64_t)sorted[q - 1] : -1;
-  int64_t cur = q < nnz ? (int64_t)sorted[q] : n;
-  if (cur > n) cur = n;  // an id outside [0, n) must not turn into a write outside colptr
-  for (int64_t u = prev + 1; u <= cur; ++u) colptr[u] = q;
+                                        int64_t n, int vector_ok, int64_t* __restrict__ colptr) {
+  const int64_t q0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColptrItems;
+  if (q0 > nnz) return;
+  uint32_t k[kColptrItems];
+  if (vector_ok && q0 + kColptrItems <= nnz) {
+    const uint4 v = *reinterpret_cast<const uint4*>(sorted + q0);
+    k[0] = v.x; k[1] = v.y; k[2] = v.z; k[3] = v.w;
+  } else {
+#pragma unroll
+    for (int i = 0; i < kColptrItems; ++i) k[i] = q0 + i < nnz ? sorted[q0 + i] : 0u;
+  }
+  int64_t prev = q0 > 0 ? (int64_t)sorted[q0 - 1] : -1;
+#pragma unroll
+  for (int i = 0; i < kColptrItems; ++i) {
+    const int64_t q = q0 + i;
+    if (q > nnz) break;
+    int64_t cur = q < nnz ? (int64_t)k[i] : n;
+    const int64_t next_prev = cur;
+    if (cur > n) cur = n;  // an id outside [0, n) must not turn into a write outside colptr
+    for (int64_t u = prev + 1; u <= cur; ++u) colptr[u] = q;
+    prev = next_prev;
+  }
 }
 
 // row_info[k] = (row r with rowptr[r] <= k < rowptr[r+1], bits of 1/deg(r)) for every CSR position
@@ -282,6 +358,7 @@ __global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+inline int aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 struct Layout {
   // csc storage
@@ -354,7 +431,8 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
       // value buffers alternate so that the last pass lands in perm
       uint32_t* vals_out = ((L.passes - 1 - p) % 2 == 0) ? perm : vals_tmp;
       uint32_t* keys_out = keys_buf[p % 2];
-      digit_histogram<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, nnz, shift, L.tiles, hist);
+      digit_histogram<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, nnz, shift, L.tiles,
+                                                               aligned16(keys_in), hist);
       DG_CUDA(cudaGetLastError());
       scan_reduce<<<(unsigned)L.chunks, kScanBlock, 0, s>>>(hist, L.hist_len, sums);
       DG_CUDA(cudaGetLastError());
@@ -369,8 +447,8 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
       keys_in = keys_out;
       vals_in = vals_out;
     }
-    const unsigned b1 = (unsigned)((nnz + 1 + 255) / 256);
-    colptr_from_sorted_keys<<<b1, 256, 0, s>>>(keys_in, nnz, n, colptr);
+    const unsigned b1 = (unsigned)(((nnz + kColptrItems) / kColptrItems + 255) / 256);
+    colptr_from_sorted_keys<<<b1, 256, 0, s>>>(keys_in, nnz, n, aligned16(keys_in), colptr);
     DG_CUDA(cudaGetLastError());
     const unsigned b2 = (unsigned)((nnz + 255) / 256);
     // colptr has been derived from the sorted keys (stream order), so both key buffers, which

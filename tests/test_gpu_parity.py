@@ -46,6 +46,24 @@ def test_tiny_transpose_bit_exact(tiny, weighted):
     check_transpose(g, *host_csr(sg))
 
 
+@pytest.mark.parametrize("shift", [1, 2, 3])
+def test_transpose_with_colidx_not_16_byte_aligned(tiny, shift):
+    """The caller's colidx only has to be 4-byte aligned: the first radix pass reads it in place
+    and must not use 16-byte loads on it.  Several tiles and a ragged last one."""
+    sg = tiny
+    rowptr = sg.rowptr.to(DEV).clone()
+    rowptr[sg.n] = rowptr[sg.n - 1]            # last row emptied: the edge count gets ragged
+    nnz = int(rowptr[sg.n])
+    store = torch.empty(nnz + 4, dtype=torch.int32, device=DEV)
+    colidx = store[shift:shift + nnz]
+    colidx.copy_(sg.colidx[:nnz])
+    w = sg.edge_w[:nnz].to(DEV).clone()
+    assert colidx.data_ptr() % 16 == 4 * shift and nnz > 3 * 4096 and nnz % 4096 != 0
+    g = binding.dg_graph_create(sg.n, nnz, rowptr, colidx, w)
+    g.dg_graph_validate()
+    check_transpose(g, to_np(rowptr), to_np(colidx), to_np(w))
+
+
 @pytest.mark.parametrize("F", [64, 8, 100, 602, 256, 128, 1, 3, 6, 130, 1028])
 @pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
 @pytest.mark.parametrize("weighted", [True, False])
