@@ -43,11 +43,13 @@ def _load():
         lib = ctypes.CDLL(_LIB_PATH)
         p = ctypes.c_void_p
         i64, i32 = ctypes.c_int64, ctypes.c_int32
-        lib.oracle_ap_forward.argtypes = [i64, p, p, p, p, i32, ctypes.c_int, p, i64, p, p]
+        lib.oracle_ap_forward.argtypes = [i64, p, p, p, p, i32, ctypes.c_int, ctypes.c_int, p, i64,
+                                          p, p]
         lib.oracle_ap_forward.restype = ctypes.c_int
         lib.oracle_transpose.argtypes = [i64, i64, p, p, p, p, p, p, p]
         lib.oracle_transpose.restype = ctypes.c_int
-        lib.oracle_ap_backward.argtypes = [i64, p, p, p, p, p, i32, ctypes.c_int, p, i64, p, p]
+        lib.oracle_ap_backward.argtypes = [i64, p, p, p, p, p, i32, ctypes.c_int, ctypes.c_int, p,
+                                           i64, p, p]
         lib.oracle_ap_backward.restype = ctypes.c_int
         lib.oracle_num_threads.restype = ctypes.c_int
         lib.oracle_set_num_threads.argtypes = [ctypes.c_int]
@@ -77,12 +79,13 @@ def _ptr(a):
     return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
 
 
-def ap_forward(rowptr, colidx, edge_w, H, op, rows=None):
+def ap_forward(rowptr, colidx, edge_w, H, op, rows=None, self_loops=False):
     """Forward AP of Algorithm 1.  Returns ``(ref, mag)``: fp64 arrays of shape (rows, F).
 
     ``ref[v] = s_v * sum_k w_k H[colidx[k]]`` over the CSR row of ``v``; ``mag`` is the same
     sum over absolute values, the quantity the fp32 error bound is stated against.
-    ``rows`` selects destination vertices (all when None).
+    ``rows`` selects destination vertices (all when None).  ``self_loops`` adds ``H[v]`` to the
+    sum and 1 to the mean's divisor (the GCN aggregator of Section 5.1).
     """
     rowptr = _arr(rowptr, np.int64, "rowptr")
     colidx = _arr(colidx, np.int32, "colidx")
@@ -97,7 +100,8 @@ def ap_forward(rowptr, colidx, edge_w, H, op, rows=None):
     ref = np.empty((count, F), dtype=np.float64)
     mag = np.empty((count, F), dtype=np.float64)
     rc = _load().oracle_ap_forward(n, _ptr(rowptr), _ptr(colidx), _ptr(edge_w), _ptr(H), F,
-                                   int(op), _ptr(rows_a), count, _ptr(ref), _ptr(mag))
+                                   int(op), int(bool(self_loops)), _ptr(rows_a), count,
+                                   _ptr(ref), _ptr(mag))
     if rc != 0:
         raise ValueError(f"oracle_ap_forward: invalid argument (code {rc})")
     return ref, mag
@@ -126,10 +130,11 @@ def transpose(rowptr, colidx, edge_w=None):
     return colptr, rowidx_T, w_T, perm
 
 
-def ap_backward(rowptr, colptr, rowidx_T, w_T, dOut, op, cols=None):
+def ap_backward(rowptr, colptr, rowidx_T, w_T, dOut, op, cols=None, self_loops=False):
     """Backward AP ``dH = A^T dOut`` over the CSC.  Returns ``(ref, mag)`` like ap_forward.
 
-    ``rowptr`` is the CSR row pointer: the mean's divisor is the in-degree of the destination.
+    ``rowptr`` is the CSR row pointer: the mean's divisor is the in-degree of the destination
+    (plus 1 with ``self_loops``, which also adds the vertex's own ``dOut`` row, scaled alike).
     """
     rowptr = _arr(rowptr, np.int64, "rowptr")
     colptr = _arr(colptr, np.int64, "colptr")
@@ -145,8 +150,8 @@ def ap_backward(rowptr, colptr, rowidx_T, w_T, dOut, op, cols=None):
     ref = np.empty((count, F), dtype=np.float64)
     mag = np.empty((count, F), dtype=np.float64)
     rc = _load().oracle_ap_backward(n, _ptr(rowptr), _ptr(colptr), _ptr(rowidx_T), _ptr(w_T),
-                                    _ptr(dOut), F, int(op), _ptr(cols_a), count,
-                                    _ptr(ref), _ptr(mag))
+                                    _ptr(dOut), F, int(op), int(bool(self_loops)),
+                                    _ptr(cols_a), count, _ptr(ref), _ptr(mag))
     if rc != 0:
         raise ValueError(f"oracle_ap_backward: invalid argument (code {rc})")
     return ref, mag

@@ -2,8 +2,8 @@
 
 The paper prints no numeric AP output, so each oracle function is pinned by something other
 than itself: a dense fp64 matrix product assembled edge by edge in Python, closed-form graphs,
-the column-sum invariant, the adjoint identity, an O(n*nnz) brute-force transpose, and scipy
-as a third party.  The planted-mistake tests at the end show that the pins notice a dropped
+the column-sum invariant, the adjoint identity, an O(n*nnz) brute-force transpose, scipy
+as a third party, and, for the self-loop switch, the graph with its loops written out.  The planted-mistake tests at the end show that the pins notice a dropped
 weight, a transposed operand, a wrong divisor and an unstable sort.
 """
 import os
@@ -280,6 +280,88 @@ def test_backward_column_subset_matches_full():
     cols = np.array([59, 3, 3, 0])
     sub, _ = oracle.ap_backward(rowptr, colptr, rowidx_T, None, G, oracle.OP_MEAN, cols=cols)
     assert np.array_equal(sub, full[cols])
+
+
+# ----------------------------------------------------------------------------- self loops
+def with_explicit_self_loops(rowptr, colidx, w):
+    """The same graph with one edge v -> v of weight 1 appended to every row."""
+    n = len(rowptr) - 1
+    rows, ws = [], []
+    for v in range(n):
+        lo, hi = rowptr[v], rowptr[v + 1]
+        rows.append(list(colidx[lo:hi]) + [v])
+        ws.extend(([1.0] * (hi - lo) if w is None else list(w[lo:hi])) + [1.0])
+    rp, ci = csr_from_lists(n, rows)
+    return rp, ci, np.asarray(ws, dtype=np.float32)
+
+
+@pytest.mark.parametrize("op", [oracle.OP_SUM, oracle.OP_MEAN])
+@pytest.mark.parametrize("weighted", [False, True])
+def test_self_loops_equal_the_graph_with_the_loops_written_out(op, weighted):
+    """Forward and backward with the switch = the plain operators on A + I (a different path
+    through the oracle: there the own row is one more edge of the loop over neighbours)."""
+    rng = np.random.default_rng(21)
+    n, nnz, F = 50, 400, 5
+    rowptr, colidx = random_csr(rng, n, nnz)           # has empty rows and duplicate edges
+    w = rng.random(nnz).astype(np.float32) if weighted else None
+    H = rng.standard_normal((n, F)).astype(np.float32)
+    G = rng.standard_normal((n, F)).astype(np.float32)
+    rp2, ci2, w2 = with_explicit_self_loops(rowptr, colidx, w)
+    got, gmag = oracle.ap_forward(rowptr, colidx, w, H, op, self_loops=True)
+    want, wmag = oracle.ap_forward(rp2, ci2, w2, H, op)
+    np.testing.assert_allclose(got, want, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(gmag, wmag, rtol=1e-13, atol=1e-15)
+    colptr, rowidx_T, w_T, _ = oracle.transpose(rowptr, colidx, w)
+    cp2, ri2, wT2, _ = oracle.transpose(rp2, ci2, w2)
+    got, gmag = oracle.ap_backward(rowptr, colptr, rowidx_T, w_T, G, op, self_loops=True)
+    want, wmag = oracle.ap_backward(rp2, cp2, ri2, wT2, G, op)
+    np.testing.assert_allclose(got, want, rtol=1e-13, atol=1e-15)
+    np.testing.assert_allclose(gmag, wmag, rtol=1e-13, atol=1e-15)
+
+
+def test_gcn_aggregator_dense_and_constant_features():
+    """(sum of neighbours + own row) / (in-degree + 1), Section 5.1: against the dense product
+    (A + I) H scaled row by row; a constant feature is a fixed point on an unweighted graph,
+    isolated vertices included."""
+    rng = np.random.default_rng(22)
+    n, nnz, F = 40, 70, 4
+    rowptr, colidx = random_csr(rng, n, nnz)
+    H = rng.standard_normal((n, F)).astype(np.float32)
+    A = dense_from_csr(rowptr, colidx, None, oracle.OP_SUM)
+    deg = np.diff(rowptr).astype(np.float64)
+    assert (deg == 0).any()
+    want = (A @ H.astype(np.float64) + H) / (deg + 1.0)[:, None]
+    got, _ = oracle.ap_forward(rowptr, colidx, None, H, oracle.OP_MEAN, self_loops=True)
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+    const = np.full((n, 3), 2.5, dtype=np.float32)
+    got, mag = oracle.ap_forward(rowptr, colidx, None, const, oracle.OP_MEAN, self_loops=True)
+    np.testing.assert_allclose(got, const, rtol=1e-14)
+    np.testing.assert_allclose(mag, const, rtol=1e-14)
+    # backward: ((A + I)^T D) G with D = diag(1 / (deg + 1))
+    G = rng.standard_normal((n, F)).astype(np.float32)
+    colptr, rowidx_T, _, _ = oracle.transpose(rowptr, colidx, None)
+    got, _ = oracle.ap_backward(rowptr, colptr, rowidx_T, None, G, oracle.OP_MEAN, self_loops=True)
+    want = (A + np.eye(n)).T @ (G.astype(np.float64) / (deg + 1.0)[:, None])
+    np.testing.assert_allclose(got, want, rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("op", [oracle.OP_SUM, oracle.OP_MEAN])
+def test_adjoint_identity_with_self_loops(op):
+    rng = np.random.default_rng(23)
+    n, nnz, F = 300, 5000, 6
+    rowptr, colidx = random_csr(rng, n, nnz)
+    w = rng.random(nnz).astype(np.float32)
+    H = rng.standard_normal((n, F)).astype(np.float32)
+    G = rng.standard_normal((n, F)).astype(np.float32)
+    colptr, rowidx_T, w_T, _ = oracle.transpose(rowptr, colidx, w)
+    out, _ = oracle.ap_forward(rowptr, colidx, w, H, op, self_loops=True)
+    dH, _ = oracle.ap_backward(rowptr, colptr, rowidx_T, w_T, G, op, self_loops=True)
+    lhs = float((out * G.astype(np.float64)).sum())
+    rhs = float((H.astype(np.float64) * dH).sum())
+    assert abs(lhs - rhs) <= 1e-10 * max(1.0, abs(lhs))
+    # a backward pass that forgets the own row, or scales it by the out-degree, breaks it
+    plain, _ = oracle.ap_backward(rowptr, colptr, rowidx_T, w_T, G, op)
+    assert abs(lhs - float((H.astype(np.float64) * plain).sum())) > 1e-6 * abs(lhs)
 
 
 # ----------------------------------------------------------------------------- planted mistakes
