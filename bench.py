@@ -523,6 +523,33 @@ def main():
         b3.record(stream)
         torch.cuda.synchronize()
         del model_bf, run_bf
+        # the aggregator fused into the library's store step: a second handle over the same CSR
+        # with the "self_loops" attribute (its CSC tabulates 1/(deg+1) for the mean's backward)
+        g_self = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+        g_self.dg_graph_set_param("self_loops", 1)
+        for kv in args.set:
+            k, v = kv.split("=")
+            g_self.dg_graph_set_param(k, int(v))
+        g_self.dg_graph_transpose()
+        fused_ms = {}
+        for key, pf in (("aggregate_first", False), ("project_first", True)):
+            torch.manual_seed(1234)
+            model_f = graphsage.GraphSAGE(g_self, dims, project_first=pf,
+                                          fused_aggregator=True).to(dev)
+            run_f = graphsage.make_epoch(model_f, H, labels, train_idx)
+            for _ in range(3):
+                run_f()
+            torch.cuda.synchronize()
+            a4, b4 = ev(), ev()
+            a4.record(stream)
+            for _ in range(args.epochs):
+                loss_f = run_f()
+            b4.record(stream)
+            torch.cuda.synchronize()
+            fused_ms[key] = a4.elapsed_time(b4) / args.epochs
+            fused_ms[key + "_loss"] = float(loss_f)
+            del model_f, run_f
+        del g_self
         epoch_info = {"ms_per_epoch": ep_ms, "epochs": args.epochs, "dims": dims,
                       "project_first": {"ms_per_epoch": a2.elapsed_time(b2) / args.epochs,
                                         "aggregations": [f"{d}:{w}" for d, w in pf_calls],
@@ -530,6 +557,11 @@ def main():
                                                 "narrows; same function up to fp32 rounding",
                                         "ms_per_epoch_bf16_aggregation":
                                             a3.elapsed_time(b3) / args.epochs},
+                      "fused_aggregator": {"ms_per_epoch": fused_ms["aggregate_first"],
+                                           "ms_per_epoch_project_first": fused_ms["project_first"],
+                                           "loss": fused_ms["aggregate_first_loss"],
+                                           "note": "own row and 1/(deg+1) in the aggregation's "
+                                                   "store step (graph attribute self_loops)"},
                       "train_vertices": int(train_idx.numel()), "loss": float(last_loss),
                       "aggregations": [f"{d}:{w}" for d, w in calls],
                       "ap_edge_feat_per_epoch": sg.nnz * sum(w for _, w in calls),

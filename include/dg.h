@@ -138,6 +138,11 @@ dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t
  * Algorithm 1 starts at zero).
  *   H    device, n x F fp32 row-major, read only
  *   out  device, n x F fp32 row-major, OVERWRITTEN (no need to clear it); must not overlap H
+ * With the graph attribute "self_loops" = 1 (dg_graph_set_param) every vertex counts as its own
+ * in-neighbour with weight 1 without such edges being stored: H[v][j] joins the sum and the
+ * mean divides by deg(v) + 1.  DG_OP_MEAN is then the GCN aggregator of GraphSAGE, Section 5.1
+ * (Models and Parameters): (sum of the neighbours' rows + own row) / (in-degree + 1), in one
+ * pass, without a second read and write of the n x F matrix.
  * fp32 accumulation in a fixed order: the same call on the same data gives the same bits.
  * Asynchronous on `stream`.
  */
@@ -151,6 +156,10 @@ dg_status_t dg_aggregate_fwd(dg_graph_t g, const float* H, int32_t F, dg_op_t op
  * (the mean's 1/deg belongs to the destination vertex v_q).  Gathers over the CSC built by
  * dg_graph_transpose, without atomics, in a fixed order.  dH is OVERWRITTEN and must not
  * overlap dOut.  Returns DG_ERR_NOT_TRANSPOSED before dg_graph_transpose.
+ * With "self_loops" = 1 the term s_u * dOut[u][j] joins the sum and s_v = 1/(deg(v) + 1) for
+ * DG_OP_MEAN.  The mean's per-edge factors are tabulated by dg_graph_transpose: set
+ * "self_loops" before it; DG_OP_MEAN returns DG_ERR_NOT_TRANSPOSED if the attribute has changed
+ * since (DG_OP_SUM does not use the table).
  * Asynchronous on `stream`.
  */
 dg_status_t dg_aggregate_bwd(dg_graph_t g, const float* dOut, int32_t F, dg_op_t op, float* dH,
@@ -203,6 +212,9 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  *                      (the blocking of Algorithm 2; 0 = choose from the L2 budget, else 1, 2,
  *                      4, 8 or 16; ignored for graphs without split pointers, i.e. with fewer
  *                      than 64 edges per vertex or unsorted rows)
+ * Graph attribute (not a tuning knob: it changes the result):
+ *   "self_loops"       0 (default) or 1: every vertex is its own in-neighbour with weight 1, see
+ *                      dg_aggregate_fwd / dg_aggregate_bwd; set it before dg_graph_transpose
  * Changing "heavy_threshold" rebuilds the heavy lists on the default stream and waits for it:
  * do not change it while aggregations of this handle are in flight.
  * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.

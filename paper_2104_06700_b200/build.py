@@ -10,7 +10,8 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_HERE, "libdgagg.so")
-SOURCES = ["dg_api.cu", "dg_graph.cu", "dg_transpose.cu", "dg_aggregate.cu", "dg_static.cu", "dg_probe.cu"]
+SOURCES = ["dg_api.cu", "dg_graph.cu", "dg_transpose.cu", "dg_aggregate.cu", "dg_aggregate_self.cu",
+           "dg_static.cu", "dg_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math=false"]
 
@@ -23,7 +24,9 @@ def _stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = _sources() + [os.path.join(CSRC, "dg_internal.cuh"), os.path.join(INCLUDE, "dg.h")]
+    deps = _sources() + [os.path.join(CSRC, "dg_internal.cuh"),
+                        os.path.join(CSRC, "dg_aggregate_kernels.cuh"),
+                        os.path.join(INCLUDE, "dg.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

@@ -118,7 +118,8 @@ static dg_status_t run_forward(Graph* g, const void* H, bool bf16, int32_t F, dg
   a.mean_rows = op == DG_OP_MEAN;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, g->split_csr, (cudaStream_t)stream);
+  const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
+  return aggregate_run(g, a, sa, g->split_csr, (cudaStream_t)stream);
 }
 
 static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F, dg_op_t op,
@@ -126,6 +127,10 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   if (dg_status_t st = check_features(g, dOut, bf16 ? 2 : 4, dH, F, op)) return st;
   if (!g->transposed) {
     set_error("the backward pass needs dg_graph_transpose first");
+    return DG_ERR_NOT_TRANSPOSED;
+  }
+  if (op == DG_OP_MEAN && g->self_loops != g->self_loops_in_csc) {
+    set_error("self_loops was changed after dg_graph_transpose: transpose again");
     return DG_ERR_NOT_TRANSPOSED;
   }
   ApArgs a{};
@@ -143,7 +148,8 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   a.mean_rows = 0;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
-  return aggregate_run(g, a, g->split_csc, (cudaStream_t)stream);
+  const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
+  return aggregate_run(g, a, sa, g->split_csc, (cudaStream_t)stream);
 }
 
 }  // namespace dg
@@ -424,6 +430,11 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     g->heavy_blocks_per_sm = value;
     return DG_OK;
   }
+  if (!strcmp(name, "self_loops")) {
+    if (value != 0 && value != 1) return invalid("self_loops must be 0 or 1");
+    g->self_loops = value;
+    return DG_OK;
+  }
   if (!strcmp(name, "source_blocks")) {
     if (value != 0 && value != 1 && value != 2 && value != 4 && value != 8 && value != 16)
       return invalid("source_blocks must be 0 (automatic), 1, 2, 4, 8 or 16");
@@ -440,6 +451,7 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
   if (!strcmp(name, "rows_per_block")) { *value = g->rows_per_block; return DG_OK; }
   if (!strcmp(name, "l2_budget_mb")) { *value = g->l2_budget_bytes >> 20; return DG_OK; }
   if (!strcmp(name, "source_blocks")) { *value = g->source_blocks; return DG_OK; }
+  if (!strcmp(name, "self_loops")) { *value = g->self_loops; return DG_OK; }
   if (!strcmp(name, "heavy_blocks_per_sm")) { *value = g->heavy_blocks_per_sm; return DG_OK; }
   return invalid("unknown parameter name");
 }
@@ -448,6 +460,6 @@ int64_t dg_kernel_launch_count(void) { return g_launches.load(std::memory_order_
 
 const char* dg_last_error(void) { return g_last_error.c_str(); }
 
-const char* dg_version(void) { return "libdgagg 0.6 sm_100a"; }
+const char* dg_version(void) { return "libdgagg 0.7 sm_100a"; }
 
 }  // extern "C"

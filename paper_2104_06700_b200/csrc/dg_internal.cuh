@@ -41,7 +41,9 @@ struct dg_graph {
   const int32_t* rowidx_T = nullptr;
   const float* w_T = nullptr;
   const int32_t* perm = nullptr;
-  const float* mean_scale_T = nullptr;  // w_T[q] / deg(rowidx_T[q]): edge factor of the mean's backward
+  const float* mean_scale_T = nullptr;  // w_T[q] / (deg(rowidx_T[q]) + self_loops): edge factor of the mean's backward
+  int64_t self_loops = 0;        // 1: every vertex is its own in-neighbour with weight 1
+  int64_t self_loops_in_csc = 0; // value mean_scale_T was built with
 
   int device = 0;
   int sm_count = 148;
@@ -86,6 +88,23 @@ struct ApArgs {
   int32_t accumulate;         // source-blocked pass after the first: add to what Y holds
 };
 
+// Implicit self loops (every vertex its own neighbour with weight 1): row r also receives
+// ss_r * X[r], once (not in accumulating passes).  self_ptr is the CSR row pointer, in both
+// directions (the in-degree belongs to the vertex, not to the segment the kernel walks);
+// nullptr = no self loops.  self_mean: ss_r = 1 / (in-degree(r) + 1) instead of 1, and
+// mean_rows scales by the same factor instead of 1 / (segment length).  A parameter of its own,
+// passed only to the kernels compiled for self loops.
+struct SelfArgs {
+  const int64_t* self_ptr;
+  int32_t self_mean;
+};
+
+// One launch of the aggregation kernels in the shape aggregate_run chose (dg_aggregate.cu,
+// dg_aggregate_self.cu).
+dg_status_t launch_plain(const dg_graph* g, const ApArgs& a, int vec, int slices, cudaStream_t s);
+dg_status_t launch_with_self_loops(const dg_graph* g, const ApArgs& a, const SelfArgs& sa, int vec,
+                                   int slices, cudaStream_t s);
+
 void set_error(const std::string& msg);
 dg_status_t cuda_fail(cudaError_t e, const char* what);
 void count_launches(int64_t k);
@@ -111,6 +130,7 @@ void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
 dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s);
 
 // dg_aggregate.cu
-dg_status_t aggregate_run(const Graph* g, const ApArgs& a, const int32_t* split, cudaStream_t s);
+dg_status_t aggregate_run(const Graph* g, const ApArgs& a, const SelfArgs& sa, const int32_t* split,
+                          cudaStream_t s);
 
 }  // namespace dg

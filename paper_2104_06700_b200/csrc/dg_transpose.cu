@@ -295,15 +295,15 @@ __global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int
   }
 }
 
-// row_info[k] = (row r with rowptr[r] <= k < rowptr[r+1], bits of 1/deg(r)) for every CSR position
-// k.  A thread takes kRowItems consecutive positions: one binary search for the first, then a
+// row_info[k] = (row r with rowptr[r] <= k < rowptr[r+1], bits of 1/(deg(r) + self)) for every
+// CSR position k; self = 1 when the graph has implicit self loops, else 0.  A thread takes kRowItems consecutive positions: one binary search for the first, then a
 // galloping search forward from the previous row for each of the others (rows are usually a few
 // positions long, empty rows are skipped in doubling strides).  Searching once per perm[q] in
 // CSC order instead, with random access to rowptr, took 218 ms of the 296 ms transpose of the
 // 1.6 G-edge graph.
 constexpr int kRowItems = 8;
-__global__ void row_info_kernel(const int64_t* __restrict__ rowptr, const float* __restrict__ inv_deg,
-                                int64_t n, int64_t nnz, uint2* __restrict__ row_info) {
+__global__ void row_info_kernel(const int64_t* __restrict__ rowptr, int self, int64_t n,
+                                int64_t nnz, uint2* __restrict__ row_info) {
   const int64_t k0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kRowItems;
   if (k0 >= nnz) return;
   int64_t lo = 0, hi = n;  // invariant: rowptr[lo] <= k0 < rowptr[hi]
@@ -332,13 +332,15 @@ __global__ void row_info_kernel(const int64_t* __restrict__ rowptr, const float*
       r = lo2;
       r_end = __ldg(rowptr + r + 1);
     }
-    row_info[k] = make_uint2((uint32_t)r, __float_as_uint(__ldg(inv_deg + r)));
+    // k lies in row r, so deg(r) >= 1
+    const float inv = 1.0f / (float)(r_end - __ldg(rowptr + r) + self);
+    row_info[k] = make_uint2((uint32_t)r, __float_as_uint(inv));
   }
 }
 
 // rowidx_T[q] = row of perm[q];  w_T[q] = edge_w[perm[q]];  mean_scale_T[q] = w_T[q] (1 if
-// unweighted) / deg(row), the factor of edge q in the backward pass of the mean, so that the
-// backward kernel streams it instead of gathering 1/deg.  One 8-byte gather per edge.
+// unweighted) / (deg(row) + self), the factor of edge q in the backward pass of the mean, so that
+// the backward kernel streams it instead of gathering 1/deg.  One 8-byte gather per edge.
 __global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64_t nnz,
                                         const uint2* __restrict__ row_info,
                                         const float* __restrict__ edge_w,
@@ -455,7 +457,7 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
     // are adjacent in the scratch, are free: they hold the nnz (row, 1/deg) pairs
     uint2* row_info = reinterpret_cast<uint2*>(sb + L.keys_a_off);
     const unsigned b3 = (unsigned)(((nnz + kRowItems - 1) / kRowItems + 255) / 256);
-    row_info_kernel<<<b3, 256, 0, s>>>(g->rowptr, g->inv_deg, n, nnz, row_info);
+    row_info_kernel<<<b3, 256, 0, s>>>(g->rowptr, g->self_loops ? 1 : 0, n, nnz, row_info);
     DG_CUDA(cudaGetLastError());
     gather_rows_and_weights<<<b2, 256, 0, s>>>(perm, nnz, row_info, g->edge_w, rowidx_T, w_T,
                                                mean_scale_T);
@@ -467,6 +469,7 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
   g->perm = reinterpret_cast<const int32_t*>(perm);
   g->w_T = w_T;
   g->mean_scale_T = mean_scale_T;
+  g->self_loops_in_csc = g->self_loops;
   g->split_csc = nullptr;
   if (wants_split(n, nnz)) {
     // the columns come out of the stable sort ordered by row, so the check never fires here

@@ -6,7 +6,9 @@ hot path: per layer  z_v = (sum_{u in N(v)} h_u + h_v) / (deg(v) + 1),  h'_v = a
 (aggregate first, then the Linear: Table 8 of the paper lists the aggregation widths 100, 256,
 256 for the 3-layer model, i.e. the layers' input widths), ReLU between layers, none after the
 last, softmax cross-entropy on a training mask, Adam.  The features need no gradient, so an
-L-layer epoch runs L forward and L-1 backward aggregations.
+L-layer epoch runs L forward and L-1 backward aggregations.  With ``fused_aggregator`` the
+own row and the division are done by the library in the aggregation's store step (graph
+attribute "self_loops"), which saves the elementwise passes over the n x F matrices.
 """
 from __future__ import annotations
 
@@ -20,11 +22,17 @@ from . import binding
 class _Aggregate(torch.autograd.Function):
     """out = A H through dg_aggregate_fwd; the backward pass calls dg_aggregate_bwd.  With
     ``bf16`` the gathered matrices (H in the forward, dOut in the backward pass) are rounded to
-    bf16 first and the bf16 entry points are used; sums and results stay fp32."""
+    bf16 first and the bf16 entry points are used; sums and results stay fp32.
+
+    ``row_scale`` (n x 1, only with op = mean on a handle with self loops): the backward pass
+    multiplies dOut by it and runs the *sum* backward on the product instead of the mean
+    backward.  Both give A^T D dOut + D dOut; the sum backward needs no per-edge factor, which
+    on graphs with long rows saves more kernel time than the one elementwise pass costs."""
 
     @staticmethod
-    def forward(ctx, H: torch.Tensor, graph: "binding.Graph", op: int, bf16: bool) -> torch.Tensor:
-        ctx.graph, ctx.op, ctx.bf16 = graph, op, bf16
+    def forward(ctx, H: torch.Tensor, graph: "binding.Graph", op: int, bf16: bool,
+                row_scale) -> torch.Tensor:
+        ctx.graph, ctx.op, ctx.bf16, ctx.row_scale = graph, op, bf16, row_scale
         if bf16:
             return graph.dg_aggregate_fwd_bf16(H.contiguous().to(torch.bfloat16), op)
         return graph.dg_aggregate_fwd(H.contiguous(), op)
@@ -33,17 +41,21 @@ class _Aggregate(torch.autograd.Function):
     def backward(ctx, dOut: torch.Tensor):
         dH = None
         if ctx.needs_input_grad[0]:
+            op = ctx.op
+            if ctx.row_scale is not None:
+                dOut = dOut * ctx.row_scale
+                op = binding.DG_OP_SUM
             if ctx.bf16:
-                dH = ctx.graph.dg_aggregate_bwd_bf16(dOut.contiguous().to(torch.bfloat16), ctx.op)
+                dH = ctx.graph.dg_aggregate_bwd_bf16(dOut.contiguous().to(torch.bfloat16), op)
             else:
-                dH = ctx.graph.dg_aggregate_bwd(dOut.contiguous(), ctx.op)
-        return dH, None, None, None
+                dH = ctx.graph.dg_aggregate_bwd(dOut.contiguous(), op)
+        return dH, None, None, None, None
 
 
 def aggregate(graph: "binding.Graph", H: torch.Tensor, op: int = binding.DG_OP_SUM,
-              bf16: bool = False) -> torch.Tensor:
+              bf16: bool = False, row_scale=None) -> torch.Tensor:
     """Differentiable aggregation primitive (the graph must have been transposed)."""
-    return _Aggregate.apply(H, graph, op, bf16)
+    return _Aggregate.apply(H, graph, op, bf16, row_scale)
 
 
 class GraphSAGE(torch.nn.Module):
@@ -57,26 +69,43 @@ class GraphSAGE(torch.nn.Module):
     """
 
     def __init__(self, graph: "binding.Graph", dims: Sequence[int], project_first: bool = False,
-                 bf16_aggregate: bool = False):
+                 bf16_aggregate: bool = False, fused_aggregator: bool = False):
         super().__init__()
         self.graph = graph
         self.project_first = project_first
         self.bf16_aggregate = bf16_aggregate   # aggregate bf16-rounded activations (even widths)
+        # the whole aggregator (own row added, division by in-degree + 1) inside the library's
+        # store step, forward and backward: needs a handle whose "self_loops" attribute was set
+        # to 1 before dg_graph_transpose
+        self.fused_aggregator = fused_aggregator
+        # backward of the fused aggregator: per-edge factors tabulated by the transpose (short
+        # rows: the elementwise pass would cost more than the factors), or dOut scaled row by
+        # row and the sum backward (long rows)
+        self.scaled_backward = graph.nnz < 64 * graph.n
+        if fused_aggregator and graph.dg_graph_get_param("self_loops") != 1:
+            raise ValueError("fused_aggregator needs a graph handle with self_loops = 1")
+        if not fused_aggregator and graph.dg_graph_get_param("self_loops") != 0:
+            raise ValueError("this handle adds self loops itself: use fused_aggregator=True")
         self.lin = torch.nn.ModuleList(
             [torch.nn.Linear(dims[i], dims[i + 1]) for i in range(len(dims) - 1)])
         deg = (graph.rowptr[1:] - graph.rowptr[:-1]).to(torch.float32)
         self.register_buffer("inv_deg1", (1.0 / (deg + 1.0)).unsqueeze(1))
 
+    def _gcn(self, M: torch.Tensor) -> torch.Tensor:
+        """(sum of the neighbours' rows + own row) / (in-degree + 1)."""
+        bf = self.bf16_aggregate and M.shape[1] % 2 == 0
+        if self.fused_aggregator:
+            return aggregate(self.graph, M, binding.DG_OP_MEAN, bf,
+                             None if self.scaled_backward else self.inv_deg1)
+        return (aggregate(self.graph, M, binding.DG_OP_SUM, bf) + M) * self.inv_deg1
+
     def forward(self, H: torch.Tensor) -> torch.Tensor:
         for i, lin in enumerate(self.lin):
             if self.project_first and lin.out_features < lin.in_features:
                 P = torch.nn.functional.linear(H, lin.weight)           # bias after the mean
-                bf = self.bf16_aggregate and P.shape[1] % 2 == 0
-                H = (aggregate(self.graph, P, binding.DG_OP_SUM, bf) + P) * self.inv_deg1 + lin.bias
+                H = self._gcn(P) + lin.bias
             else:
-                bf = self.bf16_aggregate and H.shape[1] % 2 == 0
-                Z = (aggregate(self.graph, H, binding.DG_OP_SUM, bf) + H) * self.inv_deg1
-                H = lin(Z)
+                H = lin(self._gcn(H))
             if i + 1 < len(self.lin):
                 H = torch.relu(H)
         return H

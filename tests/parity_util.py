@@ -46,23 +46,28 @@ def check_transpose(g, rowptr_h, colidx_h, w_h):
     return o_colptr, o_rowidx, o_w
 
 
-def check_fwd_bwd(g, sg_host, H, G, op, csc_host, rows=None):
-    """Forward on H and backward on G against the oracle; rows=None compares every element."""
+def check_fwd_bwd(g, sg_host, H, G, op, csc_host, rows=None, self_loops=False):
+    """Forward on H and backward on G against the oracle; rows=None compares every element.
+    `self_loops` must be the handle's "self_loops" attribute (set before the transpose)."""
     rowptr_h, colidx_h, w_h = sg_host
+    assert g.dg_graph_get_param("self_loops") == int(self_loops)
     o_colptr, o_rowidx, o_w = csc_host
     out = g.dg_aggregate_fwd(H, op)
     dH = g.dg_aggregate_bwd(G, op)
     torch.cuda.synchronize()
     Hh, Gh = to_np(H), to_np(G)
     if rows is None:
-        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, Hh, op)
+        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, Hh, op, self_loops=self_loops)
         a = assert_within_bound(to_np(out), ref, mag, "fwd")
-        ref, mag = oracle.ap_backward(rowptr_h, o_colptr, o_rowidx, o_w, Gh, op)
+        ref, mag = oracle.ap_backward(rowptr_h, o_colptr, o_rowidx, o_w, Gh, op,
+                                      self_loops=self_loops)
         b = assert_within_bound(to_np(dH), ref, mag, "bwd")
     else:
         idx = torch.as_tensor(rows, device=out.device)
-        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, Hh, op, rows=rows)
+        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, Hh, op, rows=rows,
+                                     self_loops=self_loops)
         a = assert_within_bound(to_np(out[idx]), ref, mag, "fwd (sampled rows)")
-        ref, mag = oracle.ap_backward(rowptr_h, o_colptr, o_rowidx, o_w, Gh, op, cols=rows)
+        ref, mag = oracle.ap_backward(rowptr_h, o_colptr, o_rowidx, o_w, Gh, op, cols=rows,
+                                      self_loops=self_loops)
         b = assert_within_bound(to_np(dH[idx]), ref, mag, "bwd (sampled rows)")
     return a, b

@@ -25,14 +25,22 @@ def reference_forward(sg, X, weights, biases):
     return H
 
 
+@pytest.mark.parametrize("fused", [False, "table", "row_scale"])
 @pytest.mark.parametrize("project_first", [False, True])
 @pytest.mark.parametrize("dims", [[64, 32, 7], [20, 16, 16, 5]])
-def test_epoch_loss_and_gradients_match_torch_reference(dims, project_first):
+def test_epoch_loss_and_gradients_match_torch_reference(dims, project_first, fused):
     sg = synth.make("tiny", weighted=False)
     g = make_graph(sg)
+    if fused:
+        g.dg_graph_set_param("self_loops", 1)
     g.dg_graph_transpose()
     torch.manual_seed(0)
-    model = graphsage.GraphSAGE(g, dims, project_first=project_first).to(DEV)
+    model = graphsage.GraphSAGE(g, dims, project_first=project_first,
+                                fused_aggregator=bool(fused)).to(DEV)
+    if fused == "table":
+        model.scaled_backward = True       # per-edge factors of the transpose
+    elif fused == "row_scale":
+        model.scaled_backward = False      # dOut scaled row by row, then the sum backward
     X = synth.features(sg.n, dims[0], 3, DEV)
     labels = torch.randint(0, dims[-1], (sg.n,), device=DEV)
     train_idx = torch.arange(0, sg.n, 3, device=DEV)
@@ -90,3 +98,13 @@ def test_bf16_aggregation_stays_close_to_fp32():
     assert abs(losses[0][0] - losses[1][0]) <= 2e-2 * abs(losses[0][0])
     scale = float(losses[0][1].abs().max())
     assert float((losses[0][1] - losses[1][1]).abs().max()) <= 5e-2 * scale
+
+
+def test_fused_aggregator_needs_the_matching_handle():
+    sg = synth.make("tiny", weighted=False)
+    g = make_graph(sg)
+    with pytest.raises(ValueError):
+        graphsage.GraphSAGE(g, [8, 4], fused_aggregator=True)
+    g.dg_graph_set_param("self_loops", 1)
+    with pytest.raises(ValueError):
+        graphsage.GraphSAGE(g, [8, 4])

@@ -99,6 +99,54 @@ def check_sampled(g, sg, H, G, op, rows, cols):
     return worst_f, worst_b
 
 
+def check_sampled_self_loops(g, sg, H, G, op, rows, cols):
+    """check_sampled for a handle with the "self_loops" attribute.  The sub-problem keeps the k
+    sampled segments as vertices 0..k-1 with their own feature rows, followed by the vertices
+    they reference (ids renumbered to k + position), so that the oracle finds every sampled
+    vertex's own row and in-degree where its definition looks for them."""
+    colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
+    out = g.dg_aggregate_fwd(H, op)
+    k = len(rows)
+    ridx = torch.as_tensor(rows, device=DEV)
+    sp, si, sw, uniq, _ = sample_segments(sg.rowptr, sg.colidx, sg.edge_w, rows)
+    n_sub = k + uniq.numel()
+    Hs = np.concatenate([to_np(H[ridx]), to_np(H[uniq])])
+    ref, mag = oracle.ap_forward(_pad_ptr(sp, n_sub), si + k, sw, Hs, op, rows=np.arange(k),
+                                 self_loops=True)
+    assert_within_bound(to_np(out[ridx]), ref, mag, "fwd, self loops")
+    del out
+    dH = g.dg_aggregate_bwd(G, op)
+    k = len(cols)
+    cidx = torch.as_tensor(cols, device=DEV)
+    sp, si, sw, uniq, _ = sample_segments(colptr, rowidx_T, w_T, cols)
+    n_sub = k + uniq.numel()
+    Gs = np.concatenate([to_np(G[cidx]), to_np(G[uniq])])
+    # in-degrees (CSR row lengths) of the sampled vertices, then of the referenced destinations
+    deg = np.concatenate([to_np(sg.rowptr[cidx + 1] - sg.rowptr[cidx]),
+                          to_np(sg.rowptr[uniq + 1] - sg.rowptr[uniq])])
+    rp = np.zeros(n_sub + 1, dtype=np.int64)
+    rp[1:] = np.cumsum(deg)
+    ref, mag = oracle.ap_backward(rp, _pad_ptr(sp, n_sub), si + k, sw, Gs, op, cols=np.arange(k),
+                                  self_loops=True)
+    assert_within_bound(to_np(dH[cidx]), ref, mag, "bwd, self loops")
+
+
+def test_full_size_reddit_like_with_self_loops():
+    """The GCN aggregator in one pass (graph attribute "self_loops") at the benchmark's size and
+    launch configuration: source-blocked passes, the own row added once."""
+    sg = synth.make("reddit_like", device=DEV)
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+    g.dg_graph_set_param("self_loops", 1)
+    g.dg_graph_transpose()
+    colptr = g.dg_graph_get_csc()[0]
+    rows = pick_rows(sg.rowptr, sg.n, 800, 20, 17)
+    cols = pick_rows(colptr, sg.n, 800, 20, 18)
+    for F in (602, 256):
+        H, G = synth.features(sg.n, F, 81, DEV), synth.features(sg.n, F, 82, DEV)
+        for op in (binding.DG_OP_MEAN, binding.DG_OP_SUM):
+            check_sampled_self_loops(g, sg, H, G, op, rows, cols)
+
+
 @pytest.mark.parametrize("name,F,ops", [
     ("reddit_like", 602, (binding.DG_OP_MEAN,)),
     ("products_like", 100, (binding.DG_OP_SUM, binding.DG_OP_MEAN)),
