@@ -87,8 +87,9 @@ dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t
  *   w_T[q]      edge_w[perm[q]], copied bit for bit (absent when the graph is unweighted)
  * There is exactly one correct result; it is integer work and bit-exact.
  * Next to these the storage holds two internal arrays: the per-edge factor w_T[q]/deg(rowidx_T[q])
- * that the backward pass of the mean streams, and (for graphs with at least 64 edges per
- * vertex) the split pointers of the CSC for source blocking.
+ * that the backward pass of the mean streams (deg + 1 when the graph attribute "self_loops" is
+ * set at the time of this call), and (for graphs with at least 64 edges per vertex) the split
+ * pointers of the CSC for source blocking.
  *   csc_storage  device, 256-byte aligned, >= csc_bytes; holds all these arrays, is borrowed
  *                by the handle until destroy (or the next transpose) and is what
  *                dg_graph_get_csc points into
