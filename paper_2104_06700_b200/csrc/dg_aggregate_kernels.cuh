@@ -404,43 +404,45 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
     xrow[c] = reinterpret_cast<const char*>(a.X) + (size_t)(f0 + (cok[c] ? ci : 0) * VEC) * E::kBytes;
   }
 
-  // Writes one finished row: scales by 1/length for the mean, adds the row's own input row when
-  // the graph has implicit self loops and, in a later source block, what the earlier blocks
-  // left in Y.
+  // Starts a row: zero, or, on a graph with implicit self loops, the row's own input row (taken
+  // by lane group 0 only, once: not in the accumulating launches of later source blocks).  It
+  // is loaded here, ahead of the row's edges, like one more gathered row; added in the store
+  // step instead, the load changed the instruction schedule of the whole summing loop (Reddit-
+  // like F = 602 forward: 4.44 ms per launch against 4.0 ms, with the same instruction count).
+  // The own row's factor: 1, or 1/(in-degree + 1) when the edges carry the mean's tabulated
+  // factors (backward mean); the forward mean scales the whole row in the store step.
+  // (Asking a warp's own rows into L2 with prefetch instructions when the warp starts made the
+  // DRAM-bound workloads slower, Products-like F = 602 41.4 -> 51.3 ms: not done.)
+  auto start_row = [&](int64_t r, V (&acc)[CPL]) {
+#pragma unroll
+    for (int c = 0; c < CPL; ++c) zero(acc[c]);
+    if constexpr (SELF) {
+      if (grp == 0 && !(SEG && a.accumulate)) {
+        using L = typename Pack<E, VEC>::Load;
+        const float ss = (sa.self_mean && !a.mean_rows) ? self_factor(sa.self_ptr, r) : 1.0f;
+#pragma unroll
+        for (int c = 0; c < CPL; ++c)
+          if (cok[c]) fma(acc[c], ss, ldg_vec(xrow[c] + (size_t)r * row_bytes, L()));
+      }
+    }
+  };
+
+  // Writes one finished row: scales by 1/length for the mean (length + 1 with self loops: the
+  // forward segment length is the in-degree) and, in a later source block, adds what the
+  // earlier blocks left in Y.
   auto store_row = [&](int64_t r, int len, V (&acc)[CPL]) {
     if (lane < G) {
+      const float rs = !a.mean_rows ? 1.0f
+                       : SELF      ? 1.0f / (float)(len + 1)
+                                   : (len > 0 ? 1.0f / (float)len : 1.0f);
       float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
-      if constexpr (SELF) {
-        using L = typename Pack<E, VEC>::Load;
-        const float ss = sa.self_mean ? self_factor(sa.self_ptr, r) : 1.0f;
-        const bool own = !(SEG && a.accumulate);
-        // The own row's address is rebuilt from a.X here, not taken from xrow[]: nothing of the
-        // summing loop stays live for this.  A plain load: with the evict-first hint the rows of
-        // hub vertices, which other rows gather again, lost their place in L2 (Products-like
-        // F = 602: 43.0 against 41.5 ms).
-        const char* self_row = reinterpret_cast<const char*>(a.X) +
-                               ((size_t)r * (size_t)a.F + (size_t)f0) * E::kBytes;
 #pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          if (cok[c]) {
-            float* dst = orow + (c0 + c * G) * VEC;
-            if (a.mean_rows) scale(acc[c], ss);
-            if (own)
-              fma(acc[c], ss, ldg_vec(self_row + (size_t)((c0 + c * G) * VEC) * E::kBytes, L()));
-            if (SEG && a.accumulate) add(acc[c], ld_vec(dst, V()));
-            stcs_vec(dst, acc[c]);
-          }
-        }
-      } else {
-        const float rs = (a.mean_rows && len > 0) ? 1.0f / (float)len : 1.0f;
-#pragma unroll
-        for (int c = 0; c < CPL; ++c) {
-          if (cok[c]) {
-            float* dst = orow + (c0 + c * G) * VEC;
-            if (a.mean_rows) scale(acc[c], rs);
-            if (SEG && a.accumulate) add(acc[c], ld_vec(dst, V()));
-            stcs_vec(dst, acc[c]);
-          }
+      for (int c = 0; c < CPL; ++c) {
+        if (cok[c]) {
+          float* dst = orow + (c0 + c * G) * VEC;
+          if (a.mean_rows) scale(acc[c], rs);
+          if (SEG && a.accumulate) add(acc[c], ld_vec(dst, V()));
+          stcs_vec(dst, acc[c]);
         }
       }
     }
@@ -490,8 +492,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
       const int hi = __shfl_sync(kFull, my_hi, i);
       const int len = __shfl_sync(kFull, my_full, i);
       V acc[CPL];
-#pragma unroll
-      for (int c = 0; c < CPL; ++c) zero(acc[c]);
+      start_row(rb + i, acc);
       for (int b = lo; b < hi; b += 32) {
         add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
@@ -535,8 +536,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
         continue;
       }
       V acc[CPL];
-#pragma unroll
-      for (int c = 0; c < CPL; ++c) zero(acc[c]);
+      start_row(rb + i, acc);
       int p = lo;
       while (p < hi) {
         if (p - b >= 32) {  // the stream is contiguous, so this is exactly one batch ahead

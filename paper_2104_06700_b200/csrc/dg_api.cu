@@ -460,6 +460,6 @@ int64_t dg_kernel_launch_count(void) { return g_launches.load(std::memory_order_
 
 const char* dg_last_error(void) { return g_last_error.c_str(); }
 
-const char* dg_version(void) { return "libdgagg 0.7 sm_100a"; }
+const char* dg_version(void) { return "libdgagg 0.8 sm_100a"; }
 
 }  // extern "C"
