@@ -43,11 +43,11 @@ NOMINAL_HBM_GBS = 8000.0
 # summed over its launches, from the ncu captures summarised under profiles/.  Reported as
 # roofline.traffic only while the library still has the version the capture was taken with.
 NCU_TRAFFIC = {
-    ("reddit_like", 602, "mean", 1.0): {"version": "libdgagg 0.7 sm_100a", "fwd": 8.354e9, "bwd": 11.803e9},
-    ("products_like", 100, "mean", 1.0): {"version": "libdgagg 0.7 sm_100a", "fwd": 31.027e9, "bwd": 32.636e9},
-    ("papers_like", 128, "sum", 0.1): {"version": "libdgagg 0.7 sm_100a", "fwd": 28.558e9, "bwd": 74.149e9},
+    ("reddit_like", 602, "mean", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 8.352e9, "bwd": 11.809e9},
+    ("products_like", 100, "mean", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 31.028e9, "bwd": 32.700e9},
+    ("papers_like", 128, "sum", 0.1): {"version": "libdgagg 0.8 sm_100a", "fwd": 28.559e9, "bwd": 74.006e9},
     # full size is too large to capture: the scale-0.1 capture times 10 (edges and rows both x10)
-    ("papers_like", 128, "sum", 1.0): {"version": "libdgagg 0.7 sm_100a", "fwd": 285.58e9, "bwd": 741.49e9},
+    ("papers_like", 128, "sum", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 285.59e9, "bwd": 740.06e9},
 }
 
 
