@@ -411,15 +411,23 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
   // like F = 602 forward: 4.44 ms per launch against 4.0 ms, with the same instruction count).
   // The own row's factor: 1, or 1/(in-degree + 1) when the edges carry the mean's tabulated
   // factors (backward mean); the forward mean scales the whole row in the store step.
-  // (Asking a warp's own rows into L2 with prefetch instructions when the warp starts made the
-  // DRAM-bound workloads slower, Products-like F = 602 41.4 -> 51.3 ms: not done.)
-  auto start_row = [&](int64_t r, V (&acc)[CPL]) {
+  // The next row's own row is asked into L2 one row ahead (1-2.5 % on the DRAM-bound workloads,
+  // whose rows are short against a DRAM round trip).  Asking for all of a warp's own rows when
+  // the warp starts made the same workloads slower (Products-like F = 602 41.4 -> 51.3 ms).
+  auto start_row = [&](int64_t r, V (&acc)[CPL], bool more_rows) {
 #pragma unroll
     for (int c = 0; c < CPL; ++c) zero(acc[c]);
     if constexpr (SELF) {
       if (grp == 0 && !(SEG && a.accumulate)) {
         using L = typename Pack<E, VEC>::Load;
         const float ss = (sa.self_mean && !a.mean_rows) ? self_factor(sa.self_ptr, r) : 1.0f;
+        // the warp's next row will want its own row: ask it into L2 one row ahead
+        if (more_rows) {
+#pragma unroll
+          for (int c = 0; c < CPL; ++c)
+            if (cok[c])
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(xrow[c] + (size_t)(r + 1) * row_bytes));
+        }
 #pragma unroll
         for (int c = 0; c < CPL; ++c)
           if (cok[c]) fma(acc[c], ss, ldg_vec(xrow[c] + (size_t)r * row_bytes, L()));
@@ -492,7 +500,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
       const int hi = __shfl_sync(kFull, my_hi, i);
       const int len = __shfl_sync(kFull, my_full, i);
       V acc[CPL];
-      start_row(rb + i, acc);
+      start_row(rb + i, acc, i + 1 < nrows);
       for (int b = lo; b < hi; b += 32) {
         add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
@@ -536,7 +544,7 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
         continue;
       }
       V acc[CPL];
-      start_row(rb + i, acc);
+      start_row(rb + i, acc, i + 1 < nrows);
       int p = lo;
       while (p < hi) {
         if (p - b >= 32) {  // the stream is contiguous, so this is exactly one batch ahead
