@@ -523,7 +523,7 @@ def main():
         b3.record(stream)
         torch.cuda.synchronize()
         del model_bf, run_bf
-        # the aggregator fused into the library's store step: a second handle over the same CSR
+        # the aggregator fused into the library's kernels: a second handle over the same CSR
         # with the "self_loops" attribute (its CSC tabulates 1/(deg+1) for the mean's backward)
         g_self = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
         g_self.dg_graph_set_param("self_loops", 1)
@@ -560,8 +560,8 @@ def main():
                       "fused_aggregator": {"ms_per_epoch": fused_ms["aggregate_first"],
                                            "ms_per_epoch_project_first": fused_ms["project_first"],
                                            "loss": fused_ms["aggregate_first_loss"],
-                                           "note": "own row and 1/(deg+1) in the aggregation's "
-                                                   "store step (graph attribute self_loops)"},
+                                           "note": "own row and 1/(deg+1) inside the aggregation "
+                                                   "kernels (graph attribute self_loops)"},
                       "train_vertices": int(train_idx.numel()), "loss": float(last_loss),
                       "aggregations": [f"{d}:{w}" for d, w in calls],
                       "ap_edge_feat_per_epoch": sg.nnz * sum(w for _, w in calls),

@@ -584,7 +584,7 @@ __global__ void __launch_bounds__(kBlock, 6) ap_kernel_r40(const ApArgs a, const
   ap_body<E, VEC, G, CPL, SCALED, SEG, false>(a, SelfArgs{}, heavy_blocks, part);
 }
 
-// Both again for graphs with implicit self loops: the store step adds the row's own input row.
+// Both again for graphs with implicit self loops: every row also sums its own input row.
 template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
 __global__ void __launch_bounds__(kBlock) ap_kernel_self(const ApArgs a, const int heavy_blocks,
                                                          const SelfArgs sa) {

@@ -1,5 +1,5 @@
 // The aggregation kernels compiled for graphs with implicit self loops (the row's own input row
-// joins its sum in the store step): a translation unit of its own, so that the two sets build
+// joins its sum): a translation unit of its own, so that the two sets build
 // side by side and the plain kernels carry nothing of the extra epilogue.
 #include "dg_aggregate_kernels.cuh"
 

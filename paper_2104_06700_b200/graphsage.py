@@ -7,7 +7,7 @@ hot path: per layer  z_v = (sum_{u in N(v)} h_u + h_v) / (deg(v) + 1),  h'_v = a
 256 for the 3-layer model, i.e. the layers' input widths), ReLU between layers, none after the
 last, softmax cross-entropy on a training mask, Adam.  The features need no gradient, so an
 L-layer epoch runs L forward and L-1 backward aggregations.  With ``fused_aggregator`` the
-own row and the division are done by the library in the aggregation's store step (graph
+own row and the division are done by the library inside the aggregation kernels (graph
 attribute "self_loops"), which saves the elementwise passes over the n x F matrices.
 """
 from __future__ import annotations
@@ -75,7 +75,7 @@ class GraphSAGE(torch.nn.Module):
         self.project_first = project_first
         self.bf16_aggregate = bf16_aggregate   # aggregate bf16-rounded activations (even widths)
         # the whole aggregator (own row added, division by in-degree + 1) inside the library's
-        # store step, forward and backward: needs a handle whose "self_loops" attribute was set
+        # kernels, forward and backward: needs a handle whose "self_loops" attribute was set
         # to 1 before dg_graph_transpose
         self.fused_aggregator = fused_aggregator
         # backward of the fused aggregator: per-edge factors tabulated by the transpose (short
