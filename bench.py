@@ -472,12 +472,14 @@ def main():
 
     # ---------------------------------------------------------------- GraphSAGE epoch (composite)
     epoch_info = None
-    epoch_dims = {"reddit_like": [602, 256, 41], "products_like": [100, 256, 256, 47]}
+    epoch_dims = {"reddit_like": [602, 256, 41], "products_like": [100, 256, 256, 47],
+                  "papers_like": [128, 256, 256, 172]}     # reduced scales only (memory)
     if (args.epochs > 0 and args.workload in epoch_dims and not args.feat and not two_buffers
             and not bf16):
         from paper_2104_06700_b200 import graphsage
         dims = epoch_dims[args.workload]
-        frac = 0.65 if args.workload == "reddit_like" else 196615 / 2449029
+        frac = {"reddit_like": 0.65, "products_like": 196615 / 2449029,
+                "papers_like": 0.011}[args.workload]          # training share of the vertices
         torch.manual_seed(1234)
         model = graphsage.GraphSAGE(g, dims).to(dev)
         labels = torch.randint(0, dims[-1], (sg.n,), device=dev)
