@@ -41,7 +41,7 @@ typedef enum {
   DG_ERR_CUDA = 3,            /* a CUDA runtime call failed; dg_last_error() has its text   */
   DG_ERR_NOT_TRANSPOSED = 4,  /* backward pass or CSC query before dg_graph_transpose       */
   DG_ERR_WORKSPACE = 5,       /* csc_storage or scratch smaller than the workspace query    */
-  DG_ERR_INVALID_GRAPH = 6    /* dg_graph_validate found a malformed CSR                    */
+  DG_ERR_INVALID_GRAPH = 6    /* dg_graph_create or dg_graph_validate found a malformed CSR */
 } dg_status_t;
 
 /* Reducer of Table 1 ("sum"), and the sum divided by the in-degree (Section 5.1). */
@@ -59,10 +59,15 @@ typedef struct dg_graph* dg_graph_t;
  *   edge_w  device, nnz fp32 scalars (the edge feature of Eq. 1 reduced to one value per
  *           edge and broadcast over the F features), or NULL for the unary copy of Eq. 2
  * The handle BORROWS the three arrays: they must stay valid and unchanged until
- * dg_graph_destroy.  The call allocates a few small device arrays that it owns (1/in-degree
- * per vertex, the lists of heavy rows and, for graphs with at least 64 edges per vertex, 17
- * int32 split pointers per vertex for source blocking) and synchronises the device once.
- * The arrays are trusted; dg_graph_validate checks them.
+ * dg_graph_destroy.  The call allocates a few small device arrays that it owns (the lists of
+ * heavy rows and, for graphs with at least 64 edges per vertex, 17 int32 split pointers per
+ * vertex for source blocking).  It waits for the whole device before it reads the arrays (so
+ * they may have been produced on any stream) and again before it returns.
+ * The arrays are checked here, in one streaming pass (rowptr[0] = 0, rowptr non-decreasing,
+ * rowptr[n] = nnz, every colidx in [0, n)): the aggregation kernels index the feature matrix
+ * with colidx without a range check, so a malformed CSR is refused with DG_ERR_INVALID_GRAPH
+ * and no handle is made.  Arrays that are changed afterwards are the caller's responsibility;
+ * dg_graph_validate repeats the check on request.
  */
 dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
                             const int32_t* colidx, const float* edge_w, dg_graph_t* out_graph);
@@ -216,8 +221,8 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
  * Graph attribute (not a tuning knob: it changes the result):
  *   "self_loops"       0 (default) or 1: every vertex is its own in-neighbour with weight 1, see
  *                      dg_aggregate_fwd / dg_aggregate_bwd; set it before dg_graph_transpose
- * Changing "heavy_threshold" rebuilds the heavy lists on the default stream and waits for it:
- * do not change it while aggregations of this handle are in flight.
+ * Changing "heavy_threshold" waits for the whole device, rebuilds the heavy lists and waits
+ * again: a rare, synchronous call.
  * Returns DG_ERR_INVALID_ARG for an unknown name or a value out of range.
  */
 dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value);

@@ -167,6 +167,15 @@ __device__ __forceinline__ void st_smem(float* p, float2 v) { p[0] = v.x; p[1] =
 __device__ __forceinline__ void st_smem(float* p, float4 v) {
   p[0] = v.x; p[1] = v.y; p[2] = v.z; p[3] = v.w;
 }
+__device__ __forceinline__ void add_smem(float* p, float v) { p[0] += v; }
+__device__ __forceinline__ void add_smem(float* p, float2 v) { p[0] += v.x; p[1] += v.y; }
+__device__ __forceinline__ void add_smem(float* p, float4 v) {
+  p[0] += v.x; p[1] += v.y; p[2] += v.z; p[3] += v.w;
+}
+__device__ __forceinline__ void add_smem(float* p, f8 v) {
+  add_smem(p, v.lo);
+  add_smem(p + 4, v.hi);
+}
 
 // Loads the neighbour id and the per-edge factor of the edge at position b + lane of the
 // index stream (neutral values at or beyond `end`).
@@ -286,6 +295,14 @@ __device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL])
   }
 }
 
+// A warp of a heavy segment moves its register sums into its shared-memory partial every
+// kHeavyFold batches, so that no fp32 chain is longer than 32 * kHeavyFold terms however long the
+// segment is: a segment of m entries is summed as chains of at most 512 terms, whose results form
+// a second chain of m / 4096 terms per warp, and the 8 warp partials are added last.  (One
+// register chain per warp, m / 8 terms, drifts past 1e-5 of the sum of magnitudes for same-sign
+// inputs once m reaches about 10^6.)
+constexpr int kHeavyFold = 16;
+
 // Block-per-row path for the heavy segments: block x of the first `heavy_blocks` blocks takes
 // entries x, x + heavy_blocks, ... of the heavy list; its 8 warps sum interleaved 32-edge
 // batches and the partial sums are combined in shared memory in warp order.
@@ -321,27 +338,43 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const SelfArgs sa,
     V acc[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) zero(acc[c]);
+    if (lane < G) {
+#pragma unroll
+      for (int c = 0; c < CPL; ++c)
+        if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
+    }
+    // adds the warp's register sums to its partial in shared memory and starts them afresh
+    auto fold = [&]() {
+      combine_groups<VEC, G, CPL>(acc);
+      if (lane < G) {
+#pragma unroll
+        for (int c = 0; c < CPL; ++c)
+          if (cok[c]) add_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
+      }
+#pragma unroll
+      for (int c = 0; c < CPL; ++c) zero(acc[c]);
+    };
     // warp w sums batches w, w+8, ... of the segment
     int32_t cur_u, nxt_u;
     float cur_s, nxt_s;
     int b = hi - lo > warp * 32 ? lo + warp * 32 : hi;
     if (b < hi) load_batch<SCALED>(a, b, hi, lane, cur_u, cur_s);
+    int since_fold = 0;
     while (b < hi) {
       const bool more = hi - b > kBlock;
       if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
       add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
       if (!more) break;
+      if (++since_fold == kHeavyFold) {
+        fold();
+        since_fold = 0;
+      }
       b += kBlock;
       cur_u = nxt_u;
       cur_s = nxt_s;
     }
-    combine_groups<VEC, G, CPL>(acc);
-    if (lane < G) {
-#pragma unroll
-      for (int c = 0; c < CPL; ++c)
-        if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
-    }
+    fold();
     __syncthreads();
     float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
     if constexpr (SELF) {

@@ -1,5 +1,8 @@
 // The C ABI of libdgagg: argument checks, handle bookkeeping and kernel dispatch.
 // Declarations and the meaning of every argument are in include/dg.h.
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -8,42 +11,48 @@
 
 namespace dg {
 
-static thread_local std::string g_last_error;
+static thread_local char g_last_error[512] = "";
 static std::atomic<int64_t> g_launches{0};
 
-void set_error(const std::string& msg) { g_last_error = msg; }
+void set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_last_error, sizeof(g_last_error), fmt, ap);
+  va_end(ap);
+}
 
 dg_status_t cuda_fail(cudaError_t e, const char* what) {
-  g_last_error = std::string(what) + ": " + cudaGetErrorString(e);
+  set_error("%s: %s", what, cudaGetErrorString(e));
   return DG_ERR_CUDA;
 }
 
 void count_launches(int64_t k) { g_launches.fetch_add(k, std::memory_order_relaxed); }
 
 static dg_status_t invalid(const char* msg) {
-  set_error(msg);
+  set_error("%s", msg);
   return DG_ERR_INVALID_ARG;
 }
 
-static bool overlaps(const void* a, const void* b, size_t bytes) {
+// [a, a + a_bytes) and [b, b + b_bytes) share a byte
+static bool overlaps(const void* a, size_t a_bytes, const void* b, size_t b_bytes) {
   const uintptr_t x = (uintptr_t)a, y = (uintptr_t)b;
-  return x < y + bytes && y < x + bytes;
+  return x < y + b_bytes && y < x + a_bytes;
 }
 
 static dg_status_t free_owned(Graph* g) {
-  if (g->inv_deg) cudaFree(g->inv_deg);
   if (g->heavy_rows) cudaFree(g->heavy_rows);
   if (g->heavy_cols) cudaFree(g->heavy_cols);
   if (g->counters) cudaFree(g->counters);
   if (g->split_csr) cudaFree(g->split_csr);
   g->split_csr = nullptr;
-  for (cudaEvent_t e : g->aux_events) cudaEventDestroy(e);
-  g->aux_events.clear();
+  for (size_t i = 0; i < g->aux_event_count; ++i) cudaEventDestroy(g->aux_events[i]);
+  free(g->aux_events);
+  g->aux_events = nullptr;
+  g->aux_event_count = 0;
   if (g->aux_ready) {
     for (int i = 0; i < 2; ++i) cudaStreamDestroy(g->aux_stream[i]);
     g->aux_ready = false;
   }
-  g->inv_deg = nullptr;
   g->heavy_rows = g->heavy_cols = g->counters = nullptr;
   return DG_OK;
 }
@@ -152,6 +161,13 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   return aggregate_run(g, a, sa, g->split_csc, (cudaStream_t)stream);
 }
 
+static dg_status_t malformed(int flags) {
+  set_error("malformed CSR:%s%s%s%s", (flags & 1) ? " rowptr[0] != 0;" : "",
+            (flags & 2) ? " rowptr decreases;" : "", (flags & 4) ? " rowptr[n] != nnz;" : "",
+            (flags & 8) ? " colidx outside [0, n);" : "");
+  return DG_ERR_INVALID_GRAPH;
+}
+
 }  // namespace dg
 
 using namespace dg;
@@ -190,7 +206,9 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   g->heavy_cap = nnz / 64 + 1;  // enough for any threshold >= 64
   if (g->heavy_cap > n) g->heavy_cap = n > 0 ? n : 1;
 
-  e = cudaMalloc(&g->inv_deg, (size_t)(n > 0 ? n : 1) * sizeof(float));
+  // The caller may have produced the arrays on any stream: wait for the device once, then
+  // everything below runs on the default stream and is waited for before the call returns.
+  e = cudaDeviceSynchronize();
   if (e == cudaSuccess) e = cudaMalloc(&g->heavy_rows, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->counters, 4 * sizeof(int32_t));
@@ -199,15 +217,19 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
     e = cudaMalloc(&g->split_csr, (size_t)(kFineBlocks + 1) * (size_t)n * sizeof(int32_t));
   if (e != cudaSuccess) { free_owned(g); delete g; return cuda_fail(e, "cudaMalloc (graph metadata)"); }
 
-  dg_status_t st = build_degree_info(g, 0);
+  // The kernels gather X[colidx[k]] without a range check, so a malformed CSR must never reach
+  // them: one streaming pass over rowptr and colidx here (about a millisecond per 10^9 edges).
+  int flags = 0;
+  dg_status_t st = validate_csr(g, 0, &flags);
+  if (st == DG_OK && flags) st = malformed(flags);
   if (st == DG_OK) st = refresh_heavy(g, true, false, 0);
   if (st == DG_OK && g->split_csr)
     st = build_split(rowptr, colidx, n, g->fine_rows, g->split_csr, g->counters + 3, 0);
   if (st == DG_OK) {
     int32_t unsorted = 0;
     e = cudaMemcpy(&unsorted, g->counters + 3, sizeof(unsorted), cudaMemcpyDeviceToHost);
-    if (e == cudaSuccess) e = cudaStreamSynchronize(0);
-    if (e != cudaSuccess) st = cuda_fail(e, "cudaStreamSynchronize (graph create)");
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) st = cuda_fail(e, "cudaDeviceSynchronize (graph create)");
     if (st == DG_OK && unsorted && g->split_csr) {  // rows not sorted: no source blocking
       cudaFree(g->split_csr);
       g->split_csr = nullptr;
@@ -229,16 +251,7 @@ dg_status_t dg_graph_validate(dg_graph_t g, void* stream) {
   if (!g) return invalid("graph handle is NULL");
   int flags = 0;
   if (dg_status_t st = validate_csr(g, (cudaStream_t)stream, &flags)) return st;
-  if (flags) {
-    std::string m = "malformed CSR:";
-    if (flags & 1) m += " rowptr[0] != 0;";
-    if (flags & 2) m += " rowptr decreases;";
-    if (flags & 4) m += " rowptr[n] != nnz;";
-    if (flags & 8) m += " colidx outside [0, n);";
-    set_error(m);
-    return DG_ERR_INVALID_GRAPH;
-  }
-  return DG_OK;
+  return flags ? malformed(flags) : DG_OK;
 }
 
 dg_status_t dg_graph_transpose_workspace(dg_graph_t g, size_t* csc_bytes, size_t* scratch_bytes) {
@@ -260,7 +273,7 @@ dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes
     set_error("workspace smaller than dg_graph_transpose_workspace reports");
     return DG_ERR_WORKSPACE;
   }
-  if (overlaps(csc_storage, scratch, need_csc < need_scratch ? need_csc : need_scratch))
+  if (overlaps(csc_storage, need_csc, scratch, need_scratch))
     return invalid("csc_storage and scratch overlap");
   g->transposed = false;
   if (dg_status_t st = transpose_run(g, csc_storage, scratch, (cudaStream_t)stream)) return st;
@@ -315,10 +328,17 @@ static dg_status_t host_pipeline(Graph* g, size_t events) {
       DG_CUDA(cudaStreamCreateWithFlags(&g->aux_stream[i], cudaStreamNonBlocking));
     g->aux_ready = true;
   }
-  while (g->aux_events.size() < events) {
-    cudaEvent_t e;
-    DG_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-    g->aux_events.push_back(e);
+  if (g->aux_event_count < events) {
+    cudaEvent_t* grown = (cudaEvent_t*)realloc(g->aux_events, events * sizeof(cudaEvent_t));
+    if (!grown) {
+      set_error("out of host memory (event pool)");
+      return DG_ERR_INVALID_ARG;
+    }
+    g->aux_events = grown;
+    while (g->aux_event_count < events) {
+      DG_CUDA(cudaEventCreateWithFlags(&g->aux_events[g->aux_event_count], cudaEventDisableTiming));
+      ++g->aux_event_count;
+    }
   }
   return DG_OK;
 }
@@ -353,7 +373,7 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
   if (dg_status_t st = host_pipeline(g, 1 + 3 * (size_t)tasks)) return st;
   cudaStream_t s = (cudaStream_t)stream;
   cudaStream_t up = g->aux_stream[0], down = g->aux_stream[1];
-  cudaEvent_t* ev = g->aux_events.data();
+  cudaEvent_t* ev = g->aux_events;
   cudaEvent_t start = ev[0];
   auto uploaded = [&](int t) { return ev[1 + 3 * t]; };
   auto computed = [&](int t) { return ev[2 + 3 * t]; };
@@ -405,9 +425,11 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
   if (!g || !name) return invalid("graph handle or name is NULL");
   if (!strcmp(name, "heavy_threshold")) {
     if (value < 64 || value > (1 << 30)) return invalid("heavy_threshold must be in [64, 2^30]");
+    // the lists may be in use, or being built, on any stream: wait for the device on both sides
+    DG_CUDA(cudaDeviceSynchronize());
     g->heavy_threshold = value;
     if (dg_status_t st = refresh_heavy(g, true, true, 0)) return st;
-    DG_CUDA(cudaStreamSynchronize(0));
+    DG_CUDA(cudaDeviceSynchronize());
     return DG_OK;
   }
   if (!strcmp(name, "slice_features")) {
@@ -458,7 +480,7 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value) {
 
 int64_t dg_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
-const char* dg_last_error(void) { return g_last_error.c_str(); }
+const char* dg_last_error(void) { return g_last_error; }
 
 const char* dg_version(void) { return "libdgagg 0.8 sm_100a"; }
 

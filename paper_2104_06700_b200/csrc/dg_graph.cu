@@ -1,19 +1,11 @@
-// Graph ingest kernels: 1/in-degree per vertex, the lists of heavy segments, CSR validation.
-// All integer work except the reciprocal; nothing here waits on another block.
+// Graph ingest kernels: the lists of heavy segments, split pointers, CSR validation.
+// All integer work; nothing here waits on another block.
 #include "dg_internal.cuh"
 
 namespace dg {
 namespace {
 
 constexpr int kBlock = 256;
-
-__global__ void inv_deg_kernel(const int64_t* __restrict__ rowptr, int64_t n,
-                               float* __restrict__ inv_deg) {
-  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (v >= n) return;
-  const int64_t d = rowptr[v + 1] - rowptr[v];
-  inv_deg[v] = d > 0 ? 1.0f / (float)d : 0.0f;
-}
 
 // The heavy list holds every segment longer than `threshold`, longest first (in 64 length
 // classes, two per power of two): the blocks that walk it take entries x, x + B, x + 2B, ...,
@@ -120,14 +112,6 @@ __global__ void sorted_check_kernel(const int64_t* __restrict__ ptr,
 inline unsigned blocks_for(int64_t items) { return (unsigned)((items + kBlock - 1) / kBlock); }
 
 }  // namespace
-
-dg_status_t build_degree_info(Graph* g, cudaStream_t s) {
-  if (g->n == 0) return DG_OK;
-  inv_deg_kernel<<<blocks_for(g->n), kBlock, 0, s>>>(g->rowptr, g->n, g->inv_deg);
-  DG_CUDA(cudaGetLastError());
-  count_launches(1);
-  return DG_OK;
-}
 
 dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, int32_t* list,
                              int64_t cap, int32_t* count, cudaStream_t s) {

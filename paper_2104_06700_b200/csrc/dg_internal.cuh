@@ -5,8 +5,6 @@
 #include <stdint.h>
 
 #include <atomic>
-#include <string>
-#include <vector>
 
 #include "dg.h"
 
@@ -17,7 +15,6 @@ struct dg_graph {
   const int32_t* colidx = nullptr;
   const float* edge_w = nullptr;
 
-  float* inv_deg = nullptr;      // n: 1/deg(v), 0 for empty rows (the transpose folds it into mean_scale_T)
   int32_t* heavy_rows = nullptr; // CSR rows longer than heavy_threshold (forward)
   int32_t* heavy_cols = nullptr; // CSC columns longer than heavy_threshold (backward)
   int32_t* counters = nullptr;   // [0] #heavy rows, [1] #heavy cols, [2] validation flags
@@ -34,7 +31,8 @@ struct dg_graph {
   // dg_aggregate_host: helper streams (upload, download) and events, created on first use
   bool aux_ready = false;
   cudaStream_t aux_stream[2] = {nullptr, nullptr};
-  std::vector<cudaEvent_t> aux_events;
+  cudaEvent_t* aux_events = nullptr;  // malloc'ed pool, aux_event_count entries
+  size_t aux_event_count = 0;
 
   bool transposed = false;
   const int64_t* colptr = nullptr;
@@ -105,7 +103,9 @@ dg_status_t launch_plain(const dg_graph* g, const ApArgs& a, int vec, int slices
 dg_status_t launch_with_self_loops(const dg_graph* g, const ApArgs& a, const SelfArgs& sa, int vec,
                                    int slices, cudaStream_t s);
 
-void set_error(const std::string& msg);
+// Records the calling thread's last error message (printf-style, truncated to a fixed buffer:
+// nothing on an error path allocates, so nothing can throw across the C boundary).
+void set_error(const char* fmt, ...) __attribute__((format(printf, 1, 2)));
 dg_status_t cuda_fail(cudaError_t e, const char* what);
 void count_launches(int64_t k);
 
@@ -116,7 +116,6 @@ void count_launches(int64_t k);
   } while (0)
 
 // dg_graph.cu
-dg_status_t build_degree_info(Graph* g, cudaStream_t s);
 dg_status_t build_heavy_list(const int64_t* ptr, int64_t n, int64_t threshold, int32_t* list,
                              int64_t cap, int32_t* count, cudaStream_t s);
 dg_status_t validate_csr(Graph* g, cudaStream_t s, int* flags_host);

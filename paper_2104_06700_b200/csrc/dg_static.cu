@@ -10,7 +10,7 @@
 // The price is a fixed size limit and a fixed footprint: every GPU on which a process loads the
 // library carries the array below from load until exit, whether or not this entry point is
 // ever called.
-#include <mutex>
+#include <atomic>
 
 #include "dg_internal.cuh"
 
@@ -21,25 +21,31 @@ namespace {
 static __device__ __align__(256) unsigned char g_transpose_scratch[DG_TRANSPOSE_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-std::mutex g_setup_mutex;
-void* g_scratch_addr[kMaxDevices] = {};  // device address of the array, per device ordinal
+// device address of the array, per device ordinal (two threads that look it up at the same
+// time get the same answer, so a plain atomic slot per device is enough)
+std::atomic<void*> g_scratch_addr[kMaxDevices] = {};
 
 // In host code the array's name is only a handle for the runtime, not a pointer a kernel could
 // use; the device address has to be asked for, once per device, with that device current.
-dg_status_t scratch_address(void** out) {
+dg_status_t scratch_address(int graph_device, void** out) {
   int dev = 0;
   DG_CUDA(cudaGetDevice(&dev));
+  if (dev != graph_device) {
+    // the array of the current device would be paired with another device's graph arrays
+    dg::set_error("dg_graph_transpose_static: the handle was created on device %d, the current "
+                  "device is %d", graph_device, dev);
+    return DG_ERR_INVALID_ARG;
+  }
   if (dev < 0 || dev >= kMaxDevices) {
     dg::set_error("dg_graph_transpose_static: device ordinal beyond the table of 64 devices");
     return DG_ERR_UNSUPPORTED;
   }
-  std::lock_guard<std::mutex> lock(g_setup_mutex);
-  if (!g_scratch_addr[dev]) {
-    void* p = nullptr;
+  void* p = g_scratch_addr[dev].load(std::memory_order_acquire);
+  if (!p) {
     DG_CUDA(cudaGetSymbolAddress(&p, g_transpose_scratch));
-    g_scratch_addr[dev] = p;
+    g_scratch_addr[dev].store(p, std::memory_order_release);
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return DG_OK;
 }
 
@@ -58,10 +64,9 @@ extern "C" dg_status_t dg_graph_transpose_static(dg_graph_t g, void* csc_storage
   size_t need_csc = 0, need_scratch = 0;
   dg::transpose_sizes(g->n, g->nnz, g->edge_w != nullptr, &need_csc, &need_scratch);
   if (need_scratch > (size_t)DG_TRANSPOSE_STATIC_SCRATCH_BYTES) {
-    dg::set_error("dg_graph_transpose_static: this graph needs " + std::to_string(need_scratch) +
-                  " bytes of scratch, the built-in array holds " +
-                  std::to_string((size_t)DG_TRANSPOSE_STATIC_SCRATCH_BYTES) +
-                  "; use dg_graph_transpose with caller-supplied scratch");
+    dg::set_error("dg_graph_transpose_static: this graph needs %zu bytes of scratch, the built-in "
+                  "array holds %zu; use dg_graph_transpose with caller-supplied scratch",
+                  need_scratch, (size_t)DG_TRANSPOSE_STATIC_SCRATCH_BYTES);
     return DG_ERR_UNSUPPORTED;
   }
   if (csc_bytes < need_csc) {
@@ -69,7 +74,7 @@ extern "C" dg_status_t dg_graph_transpose_static(dg_graph_t g, void* csc_storage
     return DG_ERR_WORKSPACE;
   }
   void* scratch = nullptr;
-  if (dg_status_t st = scratch_address(&scratch)) return st;
+  if (dg_status_t st = scratch_address(g->device, &scratch)) return st;
   cudaStream_t s = (cudaStream_t)stream;
   // Every buffer of the sort (keys, values, histogram, chunk sums) is written in full before it
   // is read, so what an earlier call left in the array needs no clearing.

@@ -346,14 +346,16 @@ def make(name: str, device="cpu", scale: float = 1.0, seed: Optional[int] = None
     return fn(seed=seed, device=device, scale=scale, **kw)
 
 
-def features(n: int, F: int, seed: int, device="cpu") -> torch.Tensor:
-    """N(0,1) fp32 feature (or upstream-gradient) matrix of shape (n, F)."""
+def features(n: int, F: int, seed: int, device="cpu", nonneg: bool = False) -> torch.Tensor:
+    """N(0,1) fp32 feature (or upstream-gradient) matrix of shape (n, F); with ``nonneg`` its
+    absolute values (the sign pattern of activations behind a ReLU, which every layer after the
+    first aggregates: all terms of a sum then have one sign and rounding errors do not cancel)."""
     gen = _gen(seed, device)
-    if n * F <= (1 << 31):
-        return torch.randn((n, F), generator=gen, device=device, dtype=torch.float32)
     out = torch.empty((n, F), device=device, dtype=torch.float32)
     rows = max(1, (1 << 30) // F)
     for s in range(0, n, rows):
         e = min(n, s + rows)
-        out[s:e] = torch.randn((e - s, F), generator=gen, device=device, dtype=torch.float32)
+        torch.randn((e - s, F), generator=gen, device=device, dtype=torch.float32, out=out[s:e])
+        if nonneg:
+            out[s:e].abs_()
     return out

@@ -2,16 +2,18 @@
 times (default knobs).
 
 Configs 2-4 (Reddit-, Products- and Proteins-like): the CSC is compared with the oracle's stable
-counting sort in full, bit for bit; forward and backward AP are compared with the oracle on a
-sample of output rows (random rows plus the longest ones, which take the block-per-row path).
-Every output row depends only on its own CSR row (CSC column), so the oracle can compute the
-sampled rows one by one: it is given the sub-problem made of those rows, with the neighbour ids
-renumbered into the compact matrix of the rows they reference.
+counting sort in full, bit for bit, and forward and backward AP are compared with the oracle on
+every output element (a chunk of rows at a time).  The variant with implicit self loops is
+compared on a sample of output rows (random rows plus the longest ones, which take the
+block-per-row path).
 
 Config 5 (Papers-like, 1.6 G edges): the host cannot hold the oracle's inputs, so the CSC is
 checked through the properties that define it uniquely (perm is a permutation; keys
 non-decreasing along perm; perm increasing inside equal keys; colptr = key boundaries;
-rowidx_T = row of perm), evaluated with torch on the GPU, and AP on sampled rows as above.
+rowidx_T = row of perm), evaluated with torch on the GPU, and AP on sampled rows.  Every output
+row depends only on its own CSR row (CSC column), so the oracle can compute sampled rows one by
+one: it is given the sub-problem made of those rows, with the neighbour ids renumbered into the
+compact matrix of the rows they reference.
 
 Set DG_SKIP_FULL_SIZE=1 to skip these (they take a few minutes).
 """
@@ -72,33 +74,6 @@ def _pad_rows(M, n_sub):
     return out
 
 
-def check_sampled(g, sg, H, G, op, rows, cols):
-    """Forward on sampled destination rows, backward on sampled source columns.  The oracle
-    gets a sub-problem whose vertices 0..k-1 are the sampled segments (the others are empty) and
-    whose neighbour ids are renumbered into the compact matrix of referenced rows."""
-    colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
-    out = g.dg_aggregate_fwd(H, op)
-    sp, si, sw, uniq, _ = sample_segments(sg.rowptr, sg.colidx, sg.edge_w, rows)
-    n_sub = max(len(rows), uniq.numel())
-    ref, mag = oracle.ap_forward(_pad_ptr(sp, n_sub), si, sw, _pad_rows(to_np(H[uniq]), n_sub), op,
-                                 rows=np.arange(len(rows)))
-    worst_f = assert_within_bound(to_np(out[torch.as_tensor(rows, device=DEV)]), ref, mag, "fwd")
-    del out
-    dH = g.dg_aggregate_bwd(G, op)
-    sp, si, sw, uniq, _ = sample_segments(colptr, rowidx_T, w_T, cols)
-    n_sub = max(len(cols), uniq.numel())
-    # the mean's divisor belongs to the destination vertex: the oracle reads it from a CSR row
-    # pointer, here one that gives every renumbered destination its true in-degree
-    deg = to_np(sg.rowptr[uniq + 1] - sg.rowptr[uniq])
-    rp = np.zeros(n_sub + 1, dtype=np.int64)
-    rp[1:len(deg) + 1] = np.cumsum(deg)
-    rp[len(deg) + 1:] = rp[len(deg)]
-    ref, mag = oracle.ap_backward(rp, _pad_ptr(sp, n_sub), si, sw,
-                                  _pad_rows(to_np(G[uniq]), n_sub), op, cols=np.arange(len(cols)))
-    worst_b = assert_within_bound(to_np(dH[torch.as_tensor(cols, device=DEV)]), ref, mag, "bwd")
-    return worst_f, worst_b
-
-
 def check_sampled_self_loops(g, sg, H, G, op, rows, cols):
     """check_sampled for a handle with the "self_loops" attribute.  The sub-problem keeps the k
     sampled segments as vertices 0..k-1 with their own feature rows, followed by the vertices
@@ -147,38 +122,56 @@ def test_full_size_reddit_like_with_self_loops():
             check_sampled_self_loops(g, sg, H, G, op, rows, cols)
 
 
-@pytest.mark.parametrize("name,F,ops", [
-    ("reddit_like", 602, (binding.DG_OP_MEAN,)),
-    ("products_like", 100, (binding.DG_OP_SUM, binding.DG_OP_MEAN)),
-    ("proteins_like", 64, (binding.DG_OP_SUM,)),
+def check_full(g, csr_host, csc_host, H, G, op, elems_per_chunk=1 << 27):
+    """Forward on H and backward on G compared with the oracle on EVERY output element, in
+    chunks of rows so that the fp64 reference of one chunk stays near 1 GB."""
+    rowptr_h, colidx_h, w_h = csr_host
+    o_colptr, o_rowidx, o_w = csc_host
+    n, F = H.shape
+    out = g.dg_aggregate_fwd(H, op)
+    dH = g.dg_aggregate_bwd(G, op)
+    torch.cuda.synchronize()
+    Hh, Gh = to_np(H), to_np(G)
+    step = max(1, elems_per_chunk // F)
+    worst_f = worst_b = 0.0
+    for s in range(0, n, step):
+        rows = np.arange(s, min(n, s + step))
+        ref, mag = oracle.ap_forward(rowptr_h, colidx_h, w_h, Hh, op, rows=rows)
+        worst_f = max(worst_f, assert_within_bound(to_np(out[s:s + step]), ref, mag, "fwd"))
+        ref, mag = oracle.ap_backward(rowptr_h, o_colptr, o_rowidx, o_w, Gh, op, cols=rows)
+        worst_b = max(worst_b, assert_within_bound(to_np(dH[s:s + step]), ref, mag, "bwd"))
+    return worst_f, worst_b
+
+
+@pytest.mark.parametrize("name,widths,ops", [
+    ("reddit_like", (602, 256), (binding.DG_OP_MEAN,)),
+    ("products_like", (100,), (binding.DG_OP_SUM, binding.DG_OP_MEAN)),
+    ("proteins_like", (8, 64, 256), (binding.DG_OP_SUM,)),
 ])
-def test_full_size_csc_bit_exact_and_sampled_rows(name, F, ops):
+def test_full_size_csc_bit_exact_and_every_output_element(name, widths, ops):
+    """Configs 2-4 at full size in the benchmark's launch configuration: the CSC bit for bit and
+    every element of the forward and the backward result against the oracle."""
     sg = synth.make(name, device=DEV)
     g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
     g.dg_graph_validate()
     g.dg_graph_transpose()
     torch.cuda.synchronize()
     colptr, rowidx_T, w_T, perm = g.dg_graph_get_csc()
-    o_colptr, o_rowidx, o_w, o_perm = oracle.transpose(
-        to_np(sg.rowptr), to_np(sg.colidx), to_np(sg.edge_w))
+    csr_host = (to_np(sg.rowptr), to_np(sg.colidx), to_np(sg.edge_w))
+    o_colptr, o_rowidx, o_w, o_perm = oracle.transpose(*csr_host)
     assert np.array_equal(to_np(colptr), o_colptr), "colptr"
     assert np.array_equal(to_np(rowidx_T), o_rowidx), "rowidx_T"
     assert np.array_equal(to_np(perm).astype(np.int64), o_perm), "perm"
     if sg.edge_w is not None:
         assert to_np(w_T).tobytes() == o_w.tobytes(), "w_T"
-    del o_colptr, o_rowidx, o_w, o_perm
-    H = synth.features(sg.n, F, 61, DEV)
-    G = synth.features(sg.n, F, 62, DEV)
-    rows = pick_rows(sg.rowptr, sg.n, 1500, 40, 7)
-    cols = pick_rows(colptr, sg.n, 1500, 40, 8)
-    for op in ops:
-        wf, wb = check_sampled(g, sg, H, G, op, rows, cols)
-        assert wf <= 1.0 and wb <= 1.0
-    # the library's widths for the other layers of the same graph
-    if name == "proteins_like":
-        for F2 in (8, 256):
-            H2, G2 = synth.features(sg.n, F2, 63, DEV), synth.features(sg.n, F2, 64, DEV)
-            check_sampled(g, sg, H2, G2, binding.DG_OP_SUM, rows[:400], cols[:400])
+    del o_perm
+    for F in widths:
+        H = synth.features(sg.n, F, 61, DEV)
+        G = synth.features(sg.n, F, 62, DEV)
+        for op in ops:
+            wf, wb = check_full(g, csr_host, (o_colptr, o_rowidx, o_w), H, G, op)
+            assert wf <= 1.0 and wb <= 1.0
+        del H, G
 
 
 def _check_csc_properties(sg, colptr, rowidx_T, perm, chunk=1 << 27):

@@ -313,19 +313,39 @@ def test_error_statuses(tiny):
     assert e.value.status == binding.DG_ERR_WORKSPACE
     with pytest.raises(binding.DgError):
         g.dg_graph_set_param("no_such_knob", 1)
-    # a malformed CSR is reported by validate, not by a fault
-    bad_col = tiny.colidx.clone().to(DEV)
-    bad_col[5] = tiny.n + 3
-    gb = binding.dg_graph_create(tiny.n, tiny.nnz, tiny.rowptr.to(DEV), bad_col, None)
-    with pytest.raises(binding.DgError) as e:
-        gb.dg_graph_validate()
-    assert e.value.status == binding.DG_ERR_INVALID_GRAPH
+    # a malformed CSR is refused at ingest (no handle is made), not found by a fault later
+    for bad_value in (tiny.n + 3, tiny.n, -1):
+        bad_col = tiny.colidx.clone().to(DEV)
+        bad_col[5] = bad_value
+        with pytest.raises(binding.DgError) as e:
+            binding.dg_graph_create(tiny.n, tiny.nnz, tiny.rowptr.to(DEV), bad_col, None)
+        assert e.value.status == binding.DG_ERR_INVALID_GRAPH and "colidx" in str(e.value)
     bad_ptr = tiny.rowptr.clone().to(DEV)
     bad_ptr[10] = bad_ptr[11] + 1
-    gp = binding.dg_graph_create(tiny.n, tiny.nnz, bad_ptr, tiny.colidx.to(DEV), None)
     with pytest.raises(binding.DgError) as e:
-        gp.dg_graph_validate()
+        binding.dg_graph_create(tiny.n, tiny.nnz, bad_ptr, tiny.colidx.to(DEV), None)
+    assert e.value.status == binding.DG_ERR_INVALID_GRAPH and "rowptr decreases" in str(e.value)
+    bad_ptr = tiny.rowptr.clone().to(DEV)
+    bad_ptr[tiny.n] -= 1
+    with pytest.raises(binding.DgError) as e:
+        binding.dg_graph_create(tiny.n, tiny.nnz, bad_ptr, tiny.colidx.to(DEV), None)
     assert e.value.status == binding.DG_ERR_INVALID_GRAPH
+    # arrays that go bad after ingest are found by dg_graph_validate
+    col = tiny.colidx.clone().to(DEV)
+    gv = binding.dg_graph_create(tiny.n, tiny.nnz, tiny.rowptr.to(DEV), col, None)
+    gv.dg_graph_validate()
+    col[7] = tiny.n
+    with pytest.raises(binding.DgError) as e:
+        gv.dg_graph_validate()
+    assert e.value.status == binding.DG_ERR_INVALID_GRAPH
+    col[7] = 0
+    # scratch inside the tail of csc_storage is an overlap, however far from its start
+    need_csc, need_scratch = g.dg_graph_transpose_workspace()
+    big = torch.empty(need_csc + need_scratch + 512, dtype=torch.uint8, device=DEV)
+    tail = ((need_csc - 256) // 256) * 256
+    with pytest.raises(binding.DgError) as e:
+        g.dg_graph_transpose(csc_storage=big[:need_csc + 256], scratch=big[tail:])
+    assert e.value.status == binding.DG_ERR_INVALID_ARG and "overlap" in str(e.value)
     # the context is still healthy
     g.dg_graph_transpose()
     g.dg_aggregate_bwd(H, binding.DG_OP_SUM)

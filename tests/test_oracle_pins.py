@@ -390,12 +390,42 @@ def test_pins_notice_planted_mistakes():
     sums, _ = oracle.ap_backward(rowptr, colptr, rowidx_T, w_T, G, oracle.OP_SUM)
     outdeg = np.maximum(np.diff(colptr), 1).astype(np.float64)
     assert not np.allclose(sums / outdeg[:, None], right)
-    # an unstable order inside one column is caught by the ordering property
+    # the five defining properties of the CSC (the check used where the oracle cannot run in
+    # full) accept the oracle's result and reject each of: an unstable order inside one column,
+    # a repeated position, a shifted column pointer, a wrong destination row
+    assert _csc_defining_properties(rowptr, colidx, colptr, rowidx_T, perm)
     u = int(np.argmax(np.diff(colptr)))
-    seg = perm[colptr[u]:colptr[u + 1]].copy()
-    assert len(seg) >= 2 and np.all(np.diff(seg) > 0)
-    seg[[0, 1]] = seg[[1, 0]]
-    assert not np.all(np.diff(seg) > 0)
+    assert colptr[u + 1] - colptr[u] >= 2
+    swapped = perm.copy()
+    swapped[[colptr[u], colptr[u] + 1]] = swapped[[colptr[u] + 1, colptr[u]]]
+    rows_swapped = rowidx_T.copy()
+    rows_swapped[[colptr[u], colptr[u] + 1]] = rows_swapped[[colptr[u] + 1, colptr[u]]]
+    assert not _csc_defining_properties(rowptr, colidx, colptr, rows_swapped, swapped)
+    repeated = perm.copy()
+    repeated[colptr[u] + 1] = repeated[colptr[u]]
+    assert not _csc_defining_properties(rowptr, colidx, colptr, rowidx_T, repeated)
+    shifted = colptr.copy()
+    shifted[u + 1] -= 1
+    assert not _csc_defining_properties(rowptr, colidx, shifted, rowidx_T, perm)
+    wrong_row = rowidx_T.copy()
+    wrong_row[colptr[u]] = (wrong_row[colptr[u]] + 1) % n
+    assert not _csc_defining_properties(rowptr, colidx, colptr, wrong_row, perm)
+
+
+def _csc_defining_properties(rowptr, colidx, colptr, rowidx_T, perm):
+    """perm is a permutation of the edge positions; the keys colidx[perm] never decrease; perm
+    increases inside equal keys; colptr holds the key boundaries; rowidx_T[q] is the CSR row
+    that contains position perm[q].  Together they admit exactly one CSC."""
+    nnz, n = len(colidx), len(rowptr) - 1
+    if sorted(perm.tolist()) != list(range(nnz)):
+        return False
+    key = colidx[perm].astype(np.int64)
+    dk = np.diff(key)
+    if np.any(dk < 0) or np.any(np.diff(perm)[dk == 0] <= 0):
+        return False
+    if not np.array_equal(colptr, np.concatenate([[0], np.cumsum(np.bincount(key, minlength=n))])):
+        return False
+    return np.array_equal(rowidx_T, np.searchsorted(rowptr, perm, side="right") - 1)
 
 
 # ----------------------------------------------------------------------------- accounting
@@ -430,8 +460,3 @@ def test_paper_accounting_values():
                                                     g["products_features"])
     assert synth.CONFIG_SHAPES["papers_like"] == (g["papers_vertices"], g["papers_edges"],
                                                   g["papers_features"])
-
-
-def test_error_bound_formula():
-    mag = np.array([0.0, 1.0, 250.0])
-    np.testing.assert_allclose(oracle.error_bound(mag), [1e-7, 1e-5 + 1e-7, 2.5e-3 + 1e-7])

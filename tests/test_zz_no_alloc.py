@@ -48,7 +48,16 @@ def test_static_scratch_transpose_matches_regular_entry_point(weighted):
     g.dg_graph_transpose_static(storage)           # first call: also looks up the array
     first = _csc_copy(g)
     storage.fill_(0xAB)                            # the second call must rewrite everything
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]     # cudaMemGetInfo: the whole device, any allocator
     g.dg_graph_transpose_static(storage)           # second call: the array holds old contents
+    torch.cuda.synchronize()
+    g.dg_graph_transpose_static(storage)           # and a later one
+    torch.cuda.synchronize()
+    # what the entry point promises: with the output storage passed in, no device memory is
+    # taken or given back by a call (nothing else runs between the two readings)
+    assert torch.cuda.mem_get_info()[0] == free_before
+    assert binding.dg_last_error() == "" or "static" not in binding.dg_last_error()
     second = _csc_copy(g)
     _same(first, want)
     _same(second, want)
