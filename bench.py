@@ -10,13 +10,17 @@ training, where the graph is static over epochs); they are timed separately and 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
                   [--workload NAME] [--scale S] [--feat F] [--op sum|mean] [--dtype f32|bf16]
                   [--set knob=value ...] [--sorted-ids] [--epochs E] [--e2e-steps S]
-                  [--no-cpu-baseline] [--no-probe]
+                  [--no-cpu-baseline] [--no-probe] [--workloads all|none]
   python bench.py --probe        # only the gather ceilings of this GPU
 
 Beside the device-resident step the line carries: the roofline object of the slower of the two
 calls (compulsory bytes, DRAM traffic from the ncu captures, gather ceilings measured in the
 same run), the same step end to end from pinned host memory ("e2e"), the CPU oracle on a row
-sample ("cpu_baseline"), and the time of one full-batch GraphSAGE epoch ("epoch").
+sample ("cpu_baseline"), the time of one full-batch GraphSAGE epoch ("epoch"), and, in the
+default run on one GPU, "workloads": one record per workload shape of the paper's Table 2 at
+full size (the tiny graph, Reddit-like at both layer widths, Products-like, Proteins-like at
+three widths, Papers-like), each with forward and backward times, compulsory bytes, roofline
+fractions, its own clock record and a sampled CPU-oracle time.
 
 N > 1 (under torchrun): the path has no exchange step and is not sharded, so every rank runs
 an independent replica of the same workload; the value is the units all ranks processed over
@@ -39,16 +43,38 @@ if ROOT not in sys.path:
 METRIC = "ap_fwd_bwd_edge_feat_per_s"
 UNIT = "edge*feat/s"
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one dg_aggregate_fwd / _bwd call,
-# summed over its launches, from the ncu captures summarised under profiles/.  Reported as
-# roofline.traffic only while the library still has the version the capture was taken with.
-NCU_TRAFFIC = {
-    ("reddit_like", 602, "mean", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 8.352e9, "bwd": 11.809e9},
-    ("products_like", 100, "mean", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 31.028e9, "bwd": 32.700e9},
-    ("papers_like", 128, "sum", 0.1): {"version": "libdgagg 0.8 sm_100a", "fwd": 28.559e9, "bwd": 74.006e9},
-    # full size is too large to capture: the scale-0.1 capture times 10 (edges and rows both x10)
-    ("papers_like", 128, "sum", 1.0): {"version": "libdgagg 0.8 sm_100a", "fwd": 285.59e9, "bwd": 740.06e9},
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+KERNEL_SOURCES = ["dg_aggregate_kernels.cuh", "dg_aggregate.cu", "dg_internal.cuh"]
+
+
+def kernel_source_hash():
+    """sha256 over the sources of the aggregation kernels: a capture is only quoted for the
+    kernels it was taken with."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2104_06700_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload, F, op, scale, direction):
+    """DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one dg_aggregate_fwd / _bwd
+    call, summed over its launches, from the ncu captures whose figures are kept in
+    profiles/dram_traffic.txt (the same file the tables under profiles/ quote).  None when no
+    capture exists for the workload or the kernel sources have changed since it was taken."""
+    if not os.path.exists(TRAFFIC_FILE):
+        return None
+    want_hash = kernel_source_hash()
+    with open(TRAFFIC_FILE) as f:
+        for line in f:
+            t = line.split("#")[0].split()
+            if len(t) != 8:
+                continue
+            wl, f_, op_, sc, src_hash, fwd, bwd, factor = t
+            if (wl, int(f_), op_, float(sc)) == (workload, F, op, float(scale)) and src_hash == want_hash:
+                return float({"fwd": fwd, "bwd": bwd}[direction]) * float(factor)
+    return None
 
 
 def parse_args():
@@ -77,6 +103,15 @@ def parse_args():
     ap.add_argument("--sorted-ids", action="store_true",
                     help="keep the generator's construction order of vertex ids (communities "
                          "contiguous) instead of a random permutation; reported separately")
+    ap.add_argument("--reorder", default="none", choices=["none", "out_degree", "in_degree"],
+                    help="rename the vertices hub-first with dg_graph_reorder before the run "
+                         "(reported separately; combine with --set hub_rows=N for the hub pass)")
+    ap.add_argument("--other-calls", action="store_true",
+                    help="also time dg_aggregate_edge_grad and two dg_ap_fwd operator pairs on "
+                         "the chosen workload (the default run does so on two workloads)")
+    ap.add_argument("--workloads", default="all", choices=["all", "none"],
+                    help="all: after the headline step, one record per workload shape at full "
+                         "size (default run on one GPU only); none: the headline alone")
     ap.add_argument("--set", action="append", default=[],
                     help="library knob name=value (heavy_threshold, slice_features, rows_per_block)")
     return ap.parse_args()
@@ -258,36 +293,360 @@ def probe_rate(binding, torch, dev, table_bytes, row_floats, count=1 << 25, reps
 
 
 def run_probe():
-    """Random-row gather rates from an L2-resident and from an HBM-sized table (one JSON line)."""
+    """Random-row gather rates of this GPU (one JSON line): from an L2-resident and an HBM-sized
+    table (dg_probe_gather), and from a block's own and a cluster partner's shared memory
+    (dg_probe_gather_smem), each also as bytes per clock per SM at the SM clock sampled meanwhile."""
     import torch
     from paper_2104_06700_b200 import binding
     dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(dev)
     stream = torch.cuda.current_stream()
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
     count = 1 << 26
-    sink = torch.empty(((count + 511) // 512) * 128, dtype=torch.float32, device=dev)
+    sink = torch.empty(((count + 511) // 512) * 128 + 16 * 128, dtype=torch.float32, device=dev)
     gen = torch.Generator(device=dev)
     gen.manual_seed(0)
-    out = {"probe": "dg_probe_gather", "gathers": count, "unit": "GB/s of gathered bytes"}
+    out = {"probe": "dg_probe_gather / dg_probe_gather_smem", "gathers": count,
+           "unit": "GB/s of gathered bytes; B/clk/SM at the sampled SM clock", "sms": sms}
+
+    def timed(call, label, row_bytes):
+        for _ in range(3):
+            call()
+        sampler = ClockSampler(dev.index or 0)
+        sampler.start()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        reps = 0
+        t0 = time.perf_counter()
+        while reps < 5 or time.perf_counter() - t0 < 0.5:
+            call()
+            reps += 1
+        b.record(stream)
+        torch.cuda.synchronize()
+        clk = sampler.stop()
+        gbs = count * row_bytes / (a.elapsed_time(b) / reps * 1e-3) / 1e9
+        mhz = clk.get("sm_mhz") or 0
+        out[label] = {"GBs": gbs, "sm_mhz": mhz,
+                      "B_per_clk_per_SM": gbs * 1e9 / (mhz * 1e6 * sms) if mhz else None}
+
     for label, table_bytes in (("l2_30MB", 30e6), ("hbm_16GB", 16e9)):
-        for row_floats in (128, 64, 32):
+        for row_floats in (128, 64, 32, 16, 8):
             rows = int(table_bytes // (row_floats * 4))
             table = torch.zeros((rows, row_floats), dtype=torch.float32, device=dev)
             idx = torch.randint(0, rows, (count,), generator=gen, device=dev, dtype=torch.int32)
-            for _ in range(3):
-                binding.dg_probe_gather(table, idx, sink)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize()
-            a.record(stream)
-            for _ in range(5):
-                binding.dg_probe_gather(table, idx, sink)
-            b.record(stream)
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / 5
-            out[f"{label}_row{row_floats * 4}B"] = count * row_floats * 4 / (ms * 1e-3) / 1e9
+            timed(lambda: binding.dg_probe_gather(table, idx, sink), f"{label}_row{row_floats * 4}B",
+                  row_floats * 4)
             del table, idx
             torch.cuda.empty_cache()
+    for remote in (False, True):
+        for row_floats in (128, 32, 16, 8):
+            stage_rows = (192 * 1024) // (row_floats * 4)
+            idx = torch.randint(0, stage_rows, (count,), generator=gen, device=dev, dtype=torch.int32)
+            timed(lambda: binding.dg_probe_gather_smem(row_floats, stage_rows, idx, sink, remote),
+                  f"smem_{'remote' if remote else 'local'}_192KB_row{row_floats * 4}B", row_floats * 4)
+            del idx
     print(json.dumps(out))
+
+
+def distinct_counts(torch, sg):
+    """(distinct sources referenced, non-empty rows): what the compulsory-bytes formula needs."""
+    seen = torch.zeros(sg.n, dtype=torch.bool, device=sg.colidx.device)
+    for s0 in range(0, sg.nnz, 1 << 28):
+        seen[sg.colidx[s0:s0 + (1 << 28)].long()] = True
+    n_ref = int(seen.sum())
+    del seen
+    return n_ref, int(((sg.rowptr[1:] - sg.rowptr[:-1]) > 0).sum())
+
+
+def sub_problem(torch, ptr, idx, w, seg_ids):
+    """The segments `seg_ids` of a CSR / CSC (device tensors) as a compact problem on the host:
+    (sub_ptr, neighbour ids renumbered 0..k-1, weights, device tensor of the k distinct ids)."""
+    seg = torch.as_tensor(seg_ids, device=ptr.device, dtype=torch.int64)
+    lo, lens = ptr[seg], ptr[seg + 1] - ptr[seg]
+    sub_ptr = torch.zeros(seg.numel() + 1, dtype=torch.int64, device=ptr.device)
+    torch.cumsum(lens, 0, out=sub_ptr[1:])
+    total = int(sub_ptr[-1])
+    owner = torch.repeat_interleave(torch.arange(seg.numel(), device=ptr.device), lens)
+    pos = lo[owner] + (torch.arange(total, device=ptr.device) - sub_ptr[owner])
+    uniq, inv = torch.unique(idx[pos].long(), return_inverse=True)
+    sub_w = None if w is None else w[pos].cpu().numpy()
+    return sub_ptr.cpu().numpy(), inv.to(torch.int32).cpu().numpy(), sub_w, uniq
+
+
+def oracle_sample_compact(torch, sg, csc, H, G, op_code, n_rows, seed=0):
+    """The oracle on `n_rows` sampled destination rows (forward) and as many sampled source columns
+    (backward), each given to it as a compact sub-problem, so that no full-size array has to
+    fit the host (every output row depends only on its own segment).  Only the oracle calls are
+    timed.  Returns (edge*feat processed, seconds)."""
+    import numpy as np
+    import oracle
+    colptr, rowidx_T, w_T = csc
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(sg.n, size=min(n_rows, sg.n), replace=False))
+    F = H.shape[1]
+    work, sec = 0, 0.0
+    for ptr, idx, w, X, fwd in ((sg.rowptr, sg.colidx, sg.edge_w, H, True),
+                                (colptr, rowidx_T, w_T, G, False)):
+        sp, si, sw, uniq = sub_problem(torch, ptr, idx, w, rows)
+        k = max(len(rows), uniq.numel())
+        ptr_k = np.full(k + 1, sp[-1], dtype=np.int64)
+        ptr_k[:len(sp)] = sp
+        Xk = np.zeros((k, F), dtype=np.float32)
+        Xk[:uniq.numel()] = X[uniq].float().cpu().numpy()
+        sel = np.arange(len(rows))
+        work += int(sp[-1]) * F
+        if fwd:
+            t0 = time.perf_counter()
+            oracle.ap_forward(ptr_k, si, sw, Xk, op_code, rows=sel)
+            sec += time.perf_counter() - t0
+        else:
+            # the mean's divisor is the in-degree of the destination: a CSR row pointer that
+            # gives every renumbered destination its true in-degree
+            deg = (sg.rowptr[uniq + 1] - sg.rowptr[uniq]).cpu().numpy()
+            rp = np.zeros(k + 1, dtype=np.int64)
+            rp[1:len(deg) + 1] = np.cumsum(deg)
+            rp[len(deg) + 1:] = rp[len(deg)]
+            t0 = time.perf_counter()
+            oracle.ap_backward(rp, ptr_k, si, sw, Xk, op_code, cols=sel)
+            sec += time.perf_counter() - t0
+    return work, sec
+
+
+def cpu_baseline_sampled(torch, sg, csc, H, G, op, seconds):
+    """cpu_baseline record of one workload: the oracle on a row sample of about `seconds`."""
+    import oracle
+    o_op = oracle.OP_MEAN if op == "mean" else oracle.OP_SUM
+    wk, sc = oracle_sample_compact(torch, sg, csc, H, G, o_op, 256)
+    n_rows = int(max(256, min(sg.n, seconds * 256 / max(sc, 1e-6))))
+    wk, sc = oracle_sample_compact(torch, sg, csc, H, G, o_op, n_rows, seed=1)
+    return {"value": wk / sc, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n_rows} of {sg.n} destination rows (fwd) and source columns (bwd) as "
+                      f"compact sub-problems, {sc:.1f} s, fp64 accumulation"}
+
+
+def median(xs):
+    xs = sorted(xs)
+    return xs[len(xs) // 2] if len(xs) % 2 else 0.5 * (xs[len(xs) // 2 - 1] + xs[len(xs) // 2])
+
+
+def direction_record(ms_list, comp_bytes, gather_bytes, units, peak, ceilings):
+    med, best = median(ms_list), min(ms_list)
+    r = {"ms_median": med, "ms_best": best, "compulsory_bytes": comp_bytes,
+         "GBs": comp_bytes / med / 1e6, "frac_of_measured": comp_bytes / med / 1e6 / peak,
+         "frac_of_8TBs": comp_bytes / med / 1e6 / NOMINAL_HBM_GBS,
+         "edge_feat_per_s": units / (med * 1e-3), "gather_GBs": gather_bytes / med / 1e6}
+    if ceilings:
+        r["gather_frac_of_l2_ceiling"] = r["gather_GBs"] / ceilings["l2_GBs"]
+        r["gather_frac_of_hbm_ceiling"] = r["gather_GBs"] / ceilings["hbm_GBs"]
+    return r
+
+
+def time_calls(torch, fwd_call, bwd_call, reps, flush, device_index):
+    """Times `reps` forward and backward calls, each between its own pair of CUDA events on the
+    current stream, with an L2 flush (a write larger than L2) before every call when `flush` is
+    a buffer.  SM clocks are sampled while the region runs."""
+    stream = torch.cuda.current_stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        fwd_call(); bwd_call()
+    marks = [[ev() for _ in range(4)] for _ in range(reps)]
+    sampler = ClockSampler(device_index)
+    sampler.start()
+    torch.cuda.synchronize()
+    for m in marks:
+        if flush is not None:
+            flush.zero_()
+        m[0].record(stream); fwd_call(); m[1].record(stream)
+        if flush is not None:
+            flush.zero_()
+        m[2].record(stream); bwd_call(); m[3].record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    return ([m[0].elapsed_time(m[1]) for m in marks], [m[2].elapsed_time(m[3]) for m in marks],
+            clocks)
+
+
+WORKLOAD_PLAN = [
+    # name, feature widths, ops, epoch dims (or None), training share of the vertices
+    ("tiny", (64,), ("sum", "mean"), None, None),
+    ("reddit_like", (602, 256), ("mean",), None, None),
+    ("products_like", (100, 256), ("sum", "mean"), [100, 256, 256, 47], 196615 / 2449029),
+    ("proteins_like", (8, 64, 256), ("sum",), None, None),
+    ("papers_like", (128,), ("sum",), None, None),
+]
+
+
+def time_one(torch, call, reps, flush):
+    """ms of `call` per repetition (median, best), each between its own pair of CUDA events."""
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        call()
+    marks = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(reps)]
+    torch.cuda.synchronize()
+    for a, b in marks:
+        if flush is not None:
+            flush.zero_()
+        a.record(stream); call(); b.record(stream)
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in marks]
+    return median(ms), min(ms)
+
+
+def extra_records(torch, binding, synth, name, g, sg, F, n_ref, peak, flush):
+    """The calls beyond sum / mean on one loaded graph: the edge-weight gradient (one sampled dot
+    product per edge, Section 2.2 of the paper) and the general AP of Table 1 with a full
+    |E| x F edge-feature matrix (mul / sum) and with the max reducer (copylhs / max).  Compulsory
+    bytes: index arrays, every referenced row once, the edge stream once, the output once."""
+    dev = sg.colidx.device
+    out = []
+    H = synth.features(sg.n, F, 100, dev)
+    G = synth.features(sg.n, F, 101, dev)
+    cold = sg.n * F * 4 <= 252e6
+    fl = flush if cold else None
+    idx_bytes = (sg.n + 1) * 8 + sg.nnz * 4
+
+    def rec(call_name, ms, comp, note):
+        med, best = ms
+        return {"workload": name, "F": F, "call": call_name, "ms_median": med, "ms_best": best,
+                "compulsory_bytes": comp, "GBs": comp / med / 1e6,
+                "frac_of_measured": comp / med / 1e6 / peak,
+                "edge_feat_per_s": sg.nnz * F / (med * 1e-3), "note": note,
+                "l2": "flushed before every call" if cold else "inputs larger than L2"}
+
+    dW = torch.empty(sg.nnz, dtype=torch.float32, device=dev)
+    ms = time_one(torch, lambda: g.dg_aggregate_edge_grad(H, G, binding.DG_OP_SUM, dW=dW), 10, fl)
+    out.append(rec("dg_aggregate_edge_grad (sum)", ms,
+                   idx_bytes + n_ref * F * 4 + sg.n * F * 4 + sg.nnz * 4,
+                   "dW[k] = <H[u_k], dOut[v_k]>: both rows per edge, H[u] gathered"))
+    del dW
+    fO = torch.empty_like(H)
+    arg = torch.empty((sg.n, F), dtype=torch.int32, device=dev)
+    ms = time_one(torch, lambda: g.dg_ap_fwd(H, None, binding.DG_BIN_COPY_LHS, binding.DG_RED_MAX,
+                                             fO=fO, arg=arg), 10, fl)
+    out.append(rec("dg_ap_fwd (copylhs, max) + arg", ms,
+                   idx_bytes + n_ref * F * 4 + 2 * sg.n * F * 4, "element-wise max with arg indices"))
+    del arg
+    if sg.nnz * F * 4 <= 24e9:
+        fE = torch.rand((sg.nnz, F), device=dev, dtype=torch.float32)
+        ms = time_one(torch, lambda: g.dg_ap_fwd(H, fE, binding.DG_BIN_MUL, binding.DG_RED_SUM,
+                                                 fO=fO), 10, None)
+        out.append(rec("dg_ap_fwd (mul, sum), |E| x F edge features", ms,
+                       idx_bytes + n_ref * F * 4 + sg.n * F * 4 + sg.nnz * F * 4,
+                       "the edge stream (nnz x F x 4 bytes, read once) dominates: HBM-streaming bound"))
+        del fE
+    return out
+
+
+def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_seconds, skip):
+    """One record per (workload, width, op) of WORKLOAD_PLAN at full size; `skip` names
+    (workload, F, op) triples that the caller has measured already."""
+    records, ingest, epochs, extras = [], {}, {}, []
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for name, widths, ops, dims, frac in WORKLOAD_PLAN:
+        torch.cuda.empty_cache()
+        t0 = time.perf_counter()
+        sg = synth.make(name, device=dev)
+        torch.cuda.synchronize()
+        gen_s = time.perf_counter() - t0
+        torch.cuda.empty_cache()
+        weighted = sg.edge_w is not None
+        n_ref, n_nonempty = distinct_counts(torch, sg)
+        t0 = time.perf_counter()
+        g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+        torch.cuda.synchronize()
+        create_ms = 1e3 * (time.perf_counter() - t0)
+        need_csc, need_scratch = g.dg_graph_transpose_workspace()
+        csc_buf = torch.empty(need_csc, dtype=torch.uint8, device=dev)
+        scratch = torch.empty(need_scratch, dtype=torch.uint8, device=dev)
+        g.dg_graph_transpose(csc_buf, scratch)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(torch.cuda.current_stream())
+        g.dg_graph_transpose(csc_buf, scratch)
+        e1.record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        ingest[name] = {"generate_s": gen_s, "graph_create_ms": create_ms,
+                        "transpose_ms": e0.elapsed_time(e1),
+                        "transpose_edges_per_s": sg.nnz / (e0.elapsed_time(e1) * 1e-3)}
+        del scratch
+        torch.cuda.empty_cache()
+        colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
+        for F in widths:
+            mat_bytes = sg.n * F * 4
+            two_buffers = 4 * mat_bytes > 0.6 * torch.cuda.get_device_properties(dev).total_memory
+            H = synth.features(sg.n, F, 100, dev)
+            out = torch.empty_like(H)
+            G, dH = (H, out) if two_buffers else (synth.features(sg.n, F, 101, dev),
+                                                  torch.empty_like(H))
+            cold = mat_bytes <= 252e6          # inputs that would stay L2-resident: flush
+            for op in ops:
+                if (name, F, op) in skip:
+                    continue
+                code = binding.DG_OP_MEAN if op == "mean" else binding.DG_OP_SUM
+                fwd_call = lambda: g.dg_aggregate_fwd(H, code, out=out)
+                bwd_call = lambda: g.dg_aggregate_bwd(G, code, dH=dH)
+                fwd_call(); bwd_call()
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(torch.cuda.current_stream()); fwd_call(); bwd_call()
+                b.record(torch.cuda.current_stream())
+                torch.cuda.synchronize()
+                est = max(a.elapsed_time(b), 1e-3)
+                reps = int(min(200, max(5 if est > 100 else 10, 400.0 / est)))
+                f_ms, b_ms, clocks = time_calls(torch, fwd_call, bwd_call, reps,
+                                                flush if cold else None, device_index)
+                b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False)
+                b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_nonempty, op == "mean")
+                rec = {"workload": name, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
+                       "weighted": weighted, "reps": reps,
+                       "l2": "flushed before every call (inputs fit L2)" if cold
+                             else "inputs larger than L2 (no flush needed)",
+                       "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
+                                  else "H, out, dOut, dH separate",
+                       "fwd": direction_record(f_ms, b_fwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
+                       "bwd": direction_record(b_ms, b_bwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
+                       "traffic": {"fwd": ncu_traffic(name, F, op, 1.0, "fwd"),
+                                   "bwd": ncu_traffic(name, F, op, 1.0, "bwd")},
+                       "clocks": clocks}
+                rec["cpu_baseline"] = None if cpu_seconds <= 0 else cpu_baseline_sampled(
+                    torch, sg, (colptr, rowidx_T, w_T), H, G, op, cpu_seconds)
+                records.append(rec)
+            if dims and F == dims[0]:
+                epochs[name] = epoch_plain(torch, g, sg, H, dims, frac, dev)
+            del H, out, G, dH
+            torch.cuda.empty_cache()
+            if (name, F) in (("products_like", 100), ("proteins_like", 64)):
+                extras += extra_records(torch, binding, synth, name, g, sg, F, n_ref, peak, flush)
+                torch.cuda.empty_cache()
+        del g, csc_buf, colptr, rowidx_T, w_T, sg
+        torch.cuda.empty_cache()
+    return records, ingest, epochs, extras
+
+
+def epoch_plain(torch, g, sg, H, dims, frac, dev, epochs=5):
+    """ms per full-batch GraphSAGE epoch in the paper's order (aggregate, then Linear)."""
+    from paper_2104_06700_b200 import graphsage
+    torch.manual_seed(1234)
+    model = graphsage.GraphSAGE(g, dims).to(dev)
+    labels = torch.randint(0, dims[-1], (sg.n,), device=dev)
+    train_idx = torch.nonzero(torch.rand(sg.n, device=dev) < frac).flatten()
+    run_epoch = graphsage.make_epoch(model, H, labels, train_idx)
+    for _ in range(3):
+        run_epoch()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(torch.cuda.current_stream())
+    for _ in range(epochs):
+        loss = run_epoch()
+    b.record(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    calls = graphsage.aggregation_calls(dims)
+    return {"ms_per_epoch": a.elapsed_time(b) / epochs, "epochs": epochs, "dims": dims,
+            "loss": float(loss), "train_vertices": int(train_idx.numel()),
+            "aggregations": [f"{d}:{w}" for d, w in calls],
+            "aggregator": "(sum + self) / (deg + 1), then Linear; ReLU; Adam"}
 
 
 def main():
@@ -322,13 +681,20 @@ def main():
     torch.cuda.empty_cache()
     F = args.feat or sg.F
     weighted = sg.edge_w is not None
-    n_ref = 0                                   # distinct sources referenced (chunked count)
-    seen = torch.zeros(sg.n, dtype=torch.bool, device=dev)
-    for s0 in range(0, sg.nnz, 1 << 28):
-        seen[sg.colidx[s0:s0 + (1 << 28)].long()] = True
-    n_ref = int(seen.sum())
-    del seen
-    n_rows_nonempty = int(((sg.rowptr[1:] - sg.rowptr[:-1]) > 0).sum())
+    n_ref, n_rows_nonempty = distinct_counts(torch, sg)
+    reorder_ms = None
+    if args.reorder != "none":
+        g0 = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        renamed = g0.dg_graph_reorder(binding.DG_ORDER_OUT_DEGREE if args.reorder == "out_degree"
+                                      else binding.DG_ORDER_IN_DEGREE)
+        torch.cuda.synchronize()
+        reorder_ms = 1e3 * (time.perf_counter() - t0)
+        del g0
+        # the run continues on the renamed graph (the features are random either way)
+        sg.rowptr, sg.colidx, sg.edge_w = renamed.rowptr, renamed.colidx, renamed.edge_w
+        torch.cuda.empty_cache()
     mat_bytes = sg.n * F * 4
     # Four n x F matrices (H, out, dOut, dH) when they fit next to the graph; otherwise two, with
     # the backward pass reading the forward pass's input buffer and overwriting its output.
@@ -402,9 +768,9 @@ def main():
         n_launch = binding.dg_kernel_launch_count() - launches0
         clk = sampler.stop() if rank == 0 else None
         tot = marks[0].elapsed_time(marks[-1])
-        f_ms = sum(marks[2 * i].elapsed_time(marks[2 * i + 1]) for i in range(args.steps)) / args.steps
-        b_ms = sum(marks[2 * i + 1].elapsed_time(marks[2 * i + 2]) for i in range(args.steps)) / args.steps
-        return tot, f_ms, b_ms, n_launch, clk
+        f_list = [marks[2 * i].elapsed_time(marks[2 * i + 1]) for i in range(args.steps)]
+        b_list = [marks[2 * i + 1].elapsed_time(marks[2 * i + 2]) for i in range(args.steps)]
+        return tot, f_list, b_list, n_launch, clk
 
     def clocks_bad(clk):
         """Thermal or hardware slowdown, or SM clocks far below maximum with no reason given."""
@@ -414,11 +780,12 @@ def main():
         stuck = clk["sm_mhz"] < 0.7 * clk["sm_max_mhz"] and not clk["reasons"]
         return bool(bad) or stuck
 
-    total_ms, fwd_ms, bwd_ms, launches, clocks = timed_region()
+    total_ms, fwd_list, bwd_list, launches, clocks = timed_region()
     remeasured = False
     if rank == 0 and world == 1 and clocks_bad(clocks):      # rejected: measure once more
         remeasured = True
-        total_ms, fwd_ms, bwd_ms, launches, clocks = timed_region()
+        total_ms, fwd_list, bwd_list, launches, clocks = timed_region()
+    fwd_ms, bwd_ms = sum(fwd_list) / len(fwd_list), sum(bwd_list) / len(bwd_list)
     if clocks is not None:
         clocks["remeasured"] = remeasured
         clocks["rejected"] = clocks_bad(clocks)
@@ -439,9 +806,9 @@ def main():
     # handles that share of the edges and of the gathered matrix)
     per_call = max(1, round(launches / (2 * args.steps)))
     traffic = None
-    t = None if bf16 else NCU_TRAFFIC.get((args.workload, F, op, args.scale))
-    if t and t["version"] == binding.dg_version() and not args.set:
-        traffic = t[dom] / per_call
+    if not bf16 and not args.set and not args.sorted_ids and args.reorder == "none":
+        t = ncu_traffic(args.workload, F, op, args.scale, dom)
+        traffic = None if t is None else t / per_call
     roofline = {
         "bound": "hbm",
         "kernel": ("ap_kernel_r40" if (weighted or (dom == "bwd" and op == "mean")) and F >= 64
@@ -461,9 +828,11 @@ def main():
     }
 
     # what this GPU can deliver to a gather at all: the aggregation's own ceilings
+    ceilings = None
     if rank == 0 and world == 1 and not args.no_probe and not two_buffers:
         l2_c = probe_rate(binding, torch, dev, 30e6, 128)
         hbm_c = probe_rate(binding, torch, dev, 8e9, 128)
+        ceilings = {"l2_GBs": l2_c, "hbm_GBs": hbm_c}
         roofline["gather_ceilings"] = {
             "how": "dg_probe_gather, random 512-byte rows, 30 MB table (L2) and 8 GB table (HBM)",
             "l2_GBs": l2_c, "hbm_GBs": hbm_c,
@@ -602,7 +971,10 @@ def main():
 
     # ---------------------------------------------------------------- CPU baseline (rank 0, N=1)
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not two_buffers and not bf16:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and two_buffers and not bf16:
+        # the host cannot hold this workload's matrices: row sample as compact sub-problems
+        cpu = cpu_baseline_sampled(torch, sg, g.dg_graph_get_csc()[:3], H, G, op, args.cpu_seconds)
+    elif rank == 0 and world == 1 and not args.no_cpu_baseline and not bf16:
         import oracle
         colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
         host = (sg.rowptr.cpu().numpy(), sg.colidx.cpu().numpy(),
@@ -621,6 +993,38 @@ def main():
                "sample": f"{n_rows} of {sg.n} destination rows (fwd) and source columns (bwd), "
                          f"{sc:.1f} s, fp64 accumulation"}
 
+    # ---------------------------------------------------------------- every workload shape (N = 1)
+    workloads = workloads_ingest = workloads_epoch = workloads_extras = None
+    if rank == 0 and world == 1 and args.other_calls and not two_buffers:
+        flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        workloads_extras = extra_records(torch, binding, synth, args.workload, g, sg, F, n_ref, peak,
+                                         flush_buf)
+        del flush_buf
+    default_run = (args.workload == "reddit_like" and args.scale == 1.0 and not args.feat
+                   and not bf16 and not args.set and not args.sorted_ids and op == "mean"
+                   and args.reorder == "none")
+    if rank == 0 and world == 1 and args.workloads == "all" and default_run:
+        head = {"workload": args.workload, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
+                "weighted": weighted, "reps": args.steps,
+                "l2": "inputs larger than L2 (no flush needed)",
+                "buffers": "H, out, dOut, dH separate",
+                "fwd": direction_record(fwd_list, b_fwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
+                "bwd": direction_record(bwd_list, b_bwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
+                "traffic": {"fwd": ncu_traffic(args.workload, F, op, 1.0, "fwd"),
+                            "bwd": ncu_traffic(args.workload, F, op, 1.0, "bwd")},
+                "clocks": clocks, "cpu_baseline": cpu, "note": "the headline step of this line"}
+        ingest_head = {"graph_create_ms": create_ms, "transpose_ms": transpose_ms,
+                       "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3)}
+        del H, out, G, dH, g, csc, sg
+        torch.cuda.empty_cache()
+        workloads, workloads_ingest, workloads_epoch, workloads_extras = run_workloads(
+            torch, binding, synth, dev, local_rank, peak, ceilings,
+            0.0 if args.no_cpu_baseline else min(3.0, args.cpu_seconds),
+            skip={(args.workload, F, op)})
+        workloads.insert(2, head)
+        workloads_ingest[args.workload + " (headline run)"] = ingest_head
+        sg = type("Shape", (), {"n": head["n"], "nnz": head["nnz"]})()
+
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -630,6 +1034,7 @@ def main():
             "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
                        "F": F, "op": op, "weighted": weighted, "step": "fwd AP + bwd AP",
                        "replicas": world, "sorted_ids": bool(args.sorted_ids),
+                       "reorder": args.reorder,
                        "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
                        else "H, out, dOut, dH separate", "l2": "inputs larger than L2 (no flush needed)"
                        if sg.n * F * 4 > 252e6 else "inputs fit L2: warm-L2 numbers",
@@ -637,7 +1042,10 @@ def main():
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "epoch": epoch_info,
             "ingest": {"graph_create_ms": create_ms, "transpose_ms": transpose_ms,
-                       "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3) if transpose_ms else None},
+                       "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3) if transpose_ms else None,
+                       "reorder_ms": reorder_ms},
+            "workloads": workloads, "workloads_ingest": workloads_ingest,
+            "workloads_epoch": workloads_epoch, "other_calls": workloads_extras,
         }))
     if world > 1:
         dist.destroy_process_group()

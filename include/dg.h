@@ -131,6 +131,16 @@ dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes
 dg_status_t dg_graph_transpose_static(dg_graph_t g, void* csc_storage, size_t csc_bytes,
                                       void* stream);
 
+/*
+ * Learnable edge weights: after the caller has changed the values of edge_w in place (an
+ * optimiser step on them, with the gradient of dg_aggregate_edge_grad), this call copies them
+ * into the CSC again (w_T[q] = edge_w[perm[q]] and the mean's per-edge factors), so that the
+ * backward pass uses the new weights.  The forward pass reads edge_w in place and needs nothing.
+ * A no-op before dg_graph_transpose; DG_ERR_INVALID_ARG for an unweighted graph.
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_graph_update_weights(dg_graph_t g, void* stream);
+
 /* Device pointers to the CSC arrays inside csc_storage (any output pointer may be NULL).
  * *w_T is set to NULL for an unweighted graph. */
 dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t** rowidx_T,
@@ -204,6 +214,113 @@ dg_status_t dg_aggregate_host(dg_graph_t g, const float* H_host, const float* dO
                               void* device_ws, size_t device_ws_bytes, void* stream);
 
 /*
+ * Vertex reordering as graph pre-processing: the same graph with its vertices renamed, so that
+ * the rows of the feature matrix that the aggregation gathers most often form one contiguous
+ * range (the GPU counterpart of the per-block CSRs the paper builds for its cache blocking,
+ * Section 3.2; Table 3 there measures the cache reuse such a layout can exploit).
+ *   order   DG_ORDER_OUT_DEGREE  hub-first by the number of edges a vertex is the source of
+ *                                (the rows the forward pass gathers most), largest first, equal
+ *                                counts by ascending old id
+ *           DG_ORDER_IN_DEGREE   the same by in-degree (the rows the backward pass gathers most)
+ *           DG_ORDER_GIVEN       the caller's permutation (from a clustering or partitioning
+ *                                tool, or community labels it already has)
+ *   given_new_of_old  device, n int32, a permutation of 0..n-1 (DG_ORDER_GIVEN only; checked:
+ *                     DG_ERR_INVALID_ARG if it is not one)
+ * The result is exact integer work with one correct answer: old vertex v becomes new_of_old[v];
+ * new row new_of_old[v] holds the entries of old row v with every source u replaced by
+ * new_of_old[u], sorted by new source id, duplicate edges in the order of their old positions;
+ * weights follow their edges bit for bit.  Aggregating the renamed features on the renamed graph
+ * gives the renamed result: AP'(P H) = P AP(H).
+ *   storage  device, 256-byte aligned, >= storage_bytes: receives new_of_old, the new rowptr,
+ *            colidx, edge_w and pos (pos[k'] = old CSR position of new position k', the order an
+ *            edge-feature matrix must be permuted into); borrowed by the new handle until it is
+ *            destroyed
+ *   scratch  device, 256-byte aligned, >= scratch_bytes; free again when the call returns
+ *   out_graph  a new handle over the renamed CSR (the attribute "self_loops" is carried over,
+ *            tuning knobs are not); the old handle stays valid and independent
+ * Synchronous (it ends like dg_graph_create).  dg_graph_get_order returns device pointers into
+ * `storage` (any output pointer may be NULL); dg_permute_rows renames the rows of a feature
+ * matrix: out[new_of_old[v]] = in[v] (to_old = 0), or out[v] = in[new_of_old[v]] (to_old = 1,
+ * results back in the old numbering); not in place.
+ */
+typedef enum { DG_ORDER_GIVEN = 0, DG_ORDER_OUT_DEGREE = 1, DG_ORDER_IN_DEGREE = 2 } dg_order_t;
+dg_status_t dg_graph_reorder_workspace(dg_graph_t g, size_t* storage_bytes, size_t* scratch_bytes);
+dg_status_t dg_graph_reorder(dg_graph_t g, dg_order_t order, const int32_t* given_new_of_old,
+                             void* storage, size_t storage_bytes, void* scratch,
+                             size_t scratch_bytes, void* stream, dg_graph_t* out_graph);
+dg_status_t dg_graph_get_order(dg_graph_t reordered, const int32_t** new_of_old,
+                               const int64_t** rowptr, const int32_t** colidx,
+                               const float** edge_w, const int32_t** pos);
+dg_status_t dg_permute_rows(const int32_t* new_of_old, int64_t n, int32_t F, const float* in,
+                            float* out, int to_old, void* stream);
+
+/*
+ * The general aggregation primitive: every operator pair of Table 1 of the paper,
+ *   fO[v][j] = (+) over the CSR row of v of  ( fV[colidx[k]][j] (x) fE[k][j] ),   0 <= j < F
+ * (Eq. 1; with one operand absent the unary copy of Eq. 2), in the pull form of Algorithm 1.
+ *   binary  (x): copylhs (the vertex feature alone), copyrhs (the edge feature alone), add, sub,
+ *           mul, div, with x = the source vertex's feature and y = the edge's feature
+ *   reduce  (+): sum, max, min
+ *   fV      device, n x F fp32 row-major; may be NULL for copyrhs
+ *   fE      device, nnz x fE_cols fp32 row-major, row k belongs to the edge at CSR position k;
+ *           fE_cols is F (the |E| x d edge features of Section 2.1) or 1 (one scalar per edge,
+ *           broadcast over the features); may be NULL for copylhs.  The edge_w given to
+ *           dg_graph_create plays no part in these calls.
+ *   fO      device, n x F fp32, OVERWRITTEN
+ *   arg     device, n x F int32, or NULL; written for max / min only: the CSR position of the
+ *           edge whose message is the extremum
+ * The paper does not say what max / min do on a vertex without in-edges, nor how ties are
+ * resolved.  Here the extremum runs over the messages of the row only (the zero the output of
+ * Algorithm 1 starts from is not a candidate), a vertex without in-edges gets 0 and arg = -1,
+ * and among equal messages the one at the lowest edge position wins.  A message is one fp32
+ * IEEE operation on the two fp32 operands, so the result of max / min is exact and the same on
+ * every run; sums are fp32 in a fixed order.
+ * Asynchronous on `stream`.
+ */
+typedef enum {
+  DG_BIN_COPY_LHS = 0, DG_BIN_COPY_RHS = 1, DG_BIN_ADD = 2, DG_BIN_SUB = 3, DG_BIN_MUL = 4,
+  DG_BIN_DIV = 5
+} dg_binary_t;
+typedef enum { DG_RED_SUM = 0, DG_RED_MAX = 1, DG_RED_MIN = 2 } dg_reduce_t;
+
+dg_status_t dg_ap_fwd(dg_graph_t g, const float* fV, const float* fE, int32_t fE_cols, int32_t F,
+                      dg_binary_t binary, dg_reduce_t reduce, float* fO, int32_t* arg,
+                      void* stream);
+
+/*
+ * Gradients of <dg_ap_fwd(fV, fE), dO> (the paper writes no backward pass; this is calculus on
+ * the definition above).  With sel(k, j) = 1 for sum and [arg[v_k][j] == k] for max / min:
+ *   dV[u][j] = sum over the edges k out of u of  sel * dO[v_k][j] * d(x (x) y)/dx
+ *   dE[k][j] =                                   sel * dO[v_k][j] * d(x (x) y)/dy
+ * (dE summed over j when fE_cols is 1: for mul / sum that is the sampled dense-dense product
+ * <fV[u_k], dO[v_k]> of Section 2.2).  The sum for dV is a gather over the CSC with an equality
+ * test on arg, without atomics and in a fixed order, so it needs dg_graph_transpose first
+ * (DG_ERR_NOT_TRANSPOSED otherwise).
+ *   dO       device, n x F
+ *   fV, fE   the operands of the forward call (those the derivative needs must be given)
+ *   arg      the forward call's arg output; required for max / min
+ *   dV       device, n x F, OVERWRITTEN; NULL to skip (all zeros for copyrhs)
+ *   dE       device, nnz x fE_cols, OVERWRITTEN; NULL to skip; must be NULL for copylhs
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const float* fE,
+                      int32_t fE_cols, int32_t F, dg_binary_t binary, dg_reduce_t reduce,
+                      const int32_t* arg, float* dV, float* dE, void* stream);
+
+/*
+ * Gradient of <dg_aggregate_fwd(H), dOut> with respect to the scalar edge weights (message
+ * passing onto edges, Section 2.2: one sampled dot product per edge):
+ *   dW[k] = s_v * sum_j H[colidx[k]][j] * dOut[v][j]      for the edge at CSR position k into v
+ * s_v = 1 for DG_OP_SUM, 1/deg(v) for DG_OP_MEAN (deg(v) + 1 with "self_loops"; the implicit
+ * loops carry no weight and get no gradient).  Works on the CSR alone; the graph's own weights
+ * do not enter (the sum is linear in them).
+ *   H, dOut  device, n x F;   dW  device, nnz fp32, OVERWRITTEN
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_aggregate_edge_grad(dg_graph_t g, const float* H, const float* dOut, int32_t F,
+                                   dg_op_t op, float* dW, void* stream);
+
+/*
  * Tuning knobs (defaults come from the device's L2 size and SM count):
  *   "heavy_threshold"  rows longer than this are summed by a whole thread block
  *   "heavy_blocks_per_sm"  thread blocks per SM that walk the list of heavy rows (longest first)
@@ -241,6 +358,20 @@ dg_status_t dg_graph_get_param(dg_graph_t g, const char* name, int64_t* value);
  */
 dg_status_t dg_probe_gather(const float* table, int64_t rows, int32_t row_floats,
                             const int32_t* idx, int64_t count, float* sink, void* stream);
+
+/*
+ * Diagnostic: the same gather served from SHARED memory.  Every thread block (1024 threads) fills a
+ * stage of stage_rows rows of row_floats fp32 (row r holds the value r everywhere; the stage
+ * must fit 200 KiB), then each warp gathers 4096 rows named by idx (values in [0, stage_rows),
+ * clamped) and sums them.  remote = 1 runs the blocks as clusters of two and reads every row
+ * from the partner block's stage (distributed shared memory).  Timed by the caller, it says what
+ * staging a block of the gathered matrix on chip could deliver, next to the L2 figure of
+ * dg_probe_gather.
+ *   idx   device, count int32;   sink  device, 16-byte aligned, >= ceil(count / 4096) * 128 floats
+ * Asynchronous on `stream`.
+ */
+dg_status_t dg_probe_gather_smem(int32_t row_floats, int32_t stage_rows, const int32_t* idx,
+                                 int64_t count, float* sink, int32_t remote, void* stream);
 
 /* Number of kernels the library has launched from this process (all handles, all threads). */
 int64_t dg_kernel_launch_count(void);

@@ -22,13 +22,18 @@ DG_ERR_WORKSPACE = 5
 DG_ERR_INVALID_GRAPH = 6
 DG_OP_SUM = 0
 DG_OP_MEAN = 1
+DG_BIN_COPY_LHS, DG_BIN_COPY_RHS, DG_BIN_ADD, DG_BIN_SUB, DG_BIN_MUL, DG_BIN_DIV = range(6)
+DG_RED_SUM, DG_RED_MAX, DG_RED_MIN = range(3)
+DG_ORDER_GIVEN, DG_ORDER_OUT_DEGREE, DG_ORDER_IN_DEGREE = range(3)
 
 EXPORTS = [
     "dg_graph_create", "dg_graph_destroy", "dg_graph_validate", "dg_graph_transpose_workspace",
-    "dg_graph_transpose", "dg_graph_transpose_static", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
+    "dg_graph_transpose", "dg_graph_transpose_static", "dg_graph_update_weights", "dg_graph_get_csc", "dg_aggregate_fwd", "dg_aggregate_bwd",
     "dg_aggregate_fwd_bf16", "dg_aggregate_bwd_bf16",
+    "dg_ap_fwd", "dg_ap_bwd", "dg_aggregate_edge_grad",
+    "dg_graph_reorder_workspace", "dg_graph_reorder", "dg_graph_get_order", "dg_permute_rows",
     "dg_aggregate_host_workspace", "dg_aggregate_host", "dg_graph_set_param",
-    "dg_graph_get_param", "dg_probe_gather", "dg_kernel_launch_count", "dg_last_error", "dg_version",
+    "dg_graph_get_param", "dg_probe_gather", "dg_probe_gather_smem", "dg_kernel_launch_count", "dg_last_error", "dg_version",
 ]
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -59,17 +64,26 @@ def lib() -> ctypes.CDLL:
         L.dg_graph_transpose_workspace.argtypes = [p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
         L.dg_graph_transpose.argtypes = [p, p, sz, p, sz, p]
         L.dg_graph_transpose_static.argtypes = [p, p, sz, p]
+        L.dg_graph_update_weights.argtypes = [p, p]
         L.dg_graph_get_csc.argtypes = [p, pp, pp, pp, pp]
         L.dg_aggregate_fwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_bwd.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_fwd_bf16.argtypes = [p, p, i32, ctypes.c_int, p, p]
         L.dg_aggregate_bwd_bf16.argtypes = [p, p, i32, ctypes.c_int, p, p]
+        L.dg_ap_fwd.argtypes = [p, p, p, i32, i32, ctypes.c_int, ctypes.c_int, p, p, p]
+        L.dg_ap_bwd.argtypes = [p, p, p, p, i32, i32, ctypes.c_int, ctypes.c_int, p, p, p, p]
+        L.dg_aggregate_edge_grad.argtypes = [p, p, p, i32, ctypes.c_int, p, p]
+        L.dg_graph_reorder_workspace.argtypes = [p, ctypes.POINTER(sz), ctypes.POINTER(sz)]
+        L.dg_graph_reorder.argtypes = [p, ctypes.c_int, p, p, sz, p, sz, p, pp]
+        L.dg_graph_get_order.argtypes = [p, pp, pp, pp, pp, pp]
+        L.dg_permute_rows.argtypes = [p, i64, i32, p, p, ctypes.c_int, p]
         L.dg_aggregate_host_workspace.argtypes = [p, i32]
         L.dg_aggregate_host_workspace.restype = sz
         L.dg_aggregate_host.argtypes = [p, p, p, i32, ctypes.c_int, p, p, p, sz, p]
         L.dg_graph_set_param.argtypes = [p, ctypes.c_char_p, i64]
         L.dg_graph_get_param.argtypes = [p, ctypes.c_char_p, ctypes.POINTER(i64)]
         L.dg_probe_gather.argtypes = [p, i64, i32, p, i64, p, p]
+        L.dg_probe_gather_smem.argtypes = [i32, i32, p, i64, p, i32, p]
         L.dg_kernel_launch_count.restype = i64
         L.dg_last_error.restype = ctypes.c_char_p
         L.dg_version.restype = ctypes.c_char_p
@@ -122,20 +136,45 @@ def dg_probe_gather(table: torch.Tensor, idx: torch.Tensor, sink: torch.Tensor, 
                                  _dev_ptr(sink, torch.float32, "sink"), _stream(stream)))
 
 
+def dg_probe_gather_smem(row_floats: int, stage_rows: int, idx: torch.Tensor, sink: torch.Tensor,
+                         remote: bool = False, stream=None) -> None:
+    """Wraps ``dg_probe_gather_smem``: idx int32 in [0, stage_rows), sink fp32."""
+    _check(lib().dg_probe_gather_smem(int(row_floats), int(stage_rows),
+                                      _dev_ptr(idx, torch.int32, "idx"), idx.numel(),
+                                      _dev_ptr(sink, torch.float32, "sink"), int(bool(remote)),
+                                      _stream(stream)))
+
+
 def dg_graph_create(n: int, nnz: int, rowptr: torch.Tensor, colidx: torch.Tensor,
                     edge_w: Optional[torch.Tensor]) -> "Graph":
     """Wraps ``dg_graph_create``; the returned object keeps the borrowed tensors alive."""
     return Graph(n, nnz, rowptr, colidx, edge_w)
 
 
+def dg_permute_rows(new_of_old: torch.Tensor, x: torch.Tensor, to_old: bool = False,
+                    out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Wraps ``dg_permute_rows``: out[new_of_old[v]] = x[v], or out[v] = x[new_of_old[v]]."""
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib().dg_permute_rows(_dev_ptr(new_of_old, torch.int32, "new_of_old"), x.shape[0],
+                                 x.shape[1], _dev_ptr(x, torch.float32, "x"),
+                                 _dev_ptr(out, torch.float32, "out"), int(bool(to_old)),
+                                 _stream(stream)))
+    return out
+
+
 class Graph:
     """Owner of one ``dg_graph_t`` and of the torch buffers the handle borrows."""
 
-    def __init__(self, n, nnz, rowptr, colidx, edge_w):
+    def __init__(self, n, nnz, rowptr, colidx, edge_w, _adopt=None):
         self._h = ctypes.c_void_p()
         self.n, self.nnz = int(n), int(nnz)
         self.rowptr, self.colidx, self.edge_w = rowptr, colidx, edge_w
         self._csc = None
+        self._storage = None
+        if _adopt is not None:          # a handle the library made (dg_graph_reorder)
+            self._h, self._storage = _adopt
+            return
         with torch.cuda.device(rowptr.device):
             _check(lib().dg_graph_create(
                 self.n, self.nnz, _dev_ptr(rowptr, torch.int64, "rowptr"),
@@ -193,6 +232,46 @@ class Graph:
             _stream(stream)))
         self._csc = csc_storage
 
+    def dg_graph_update_weights(self, stream=None) -> None:
+        _check(lib().dg_graph_update_weights(self._h, _stream(stream)))
+
+    def dg_graph_reorder_workspace(self):
+        a, b = ctypes.c_size_t(), ctypes.c_size_t()
+        _check(lib().dg_graph_reorder_workspace(self._h, ctypes.byref(a), ctypes.byref(b)))
+        return int(a.value), int(b.value)
+
+    def dg_graph_reorder(self, order: int, given_new_of_old: Optional[torch.Tensor] = None,
+                         stream=None) -> "Graph":
+        """Returns a new Graph over the renamed CSR (its arrays are views into a storage tensor
+        the new object keeps alive); ``new.new_of_old`` and ``new.pos`` give the permutations."""
+        need_storage, need_scratch = self.dg_graph_reorder_workspace()
+        storage = torch.empty(need_storage, dtype=torch.uint8, device=self.device)
+        scratch = torch.empty(need_scratch, dtype=torch.uint8, device=self.device)
+        h = ctypes.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib().dg_graph_reorder(
+                self._h, int(order), _dev_ptr(given_new_of_old, torch.int32, "given_new_of_old"),
+                ctypes.c_void_p(storage.data_ptr()), storage.numel(),
+                ctypes.c_void_p(scratch.data_ptr()), scratch.numel(), _stream(stream),
+                ctypes.byref(h)))
+        ptrs = [ctypes.c_void_p() for _ in range(5)]
+        _check(lib().dg_graph_get_order(h, *[ctypes.byref(p) for p in ptrs]))
+        base = storage.data_ptr()
+
+        def view(p, dtype, count):
+            if not p.value:
+                return None
+            off = p.value - base
+            size = torch.empty(0, dtype=dtype).element_size() * count
+            return storage[off:off + size].view(dtype)
+
+        new = Graph(self.n, self.nnz, view(ptrs[1], torch.int64, self.n + 1),
+                    view(ptrs[2], torch.int32, self.nnz), view(ptrs[3], torch.float32, self.nnz),
+                    _adopt=(h, storage))
+        new.new_of_old = view(ptrs[0], torch.int32, self.n)
+        new.pos = view(ptrs[4], torch.int32, self.nnz)
+        return new
+
     def dg_graph_get_csc(self):
         """(colptr int64[n+1], rowidx_T int32[nnz], w_T fp32[nnz] | None, perm int32[nnz]) as
         torch views into the CSC storage."""
@@ -247,6 +326,62 @@ class Graph:
                                            int(op), _dev_ptr(dH, torch.float32, "dH"),
                                            _stream(stream)))
         return dH
+
+    def _edge_cols(self, fE, F):
+        if fE is None:
+            return 1
+        if fE.dim() != 2 or fE.shape[0] != self.nnz or fE.shape[1] not in (1, F):
+            raise ValueError("fE must be (nnz, F) or (nnz, 1)")
+        return fE.shape[1]
+
+    def dg_ap_fwd(self, fV: Optional[torch.Tensor], fE: Optional[torch.Tensor], binary: int,
+                  reduce: int, F: Optional[int] = None, fO: Optional[torch.Tensor] = None,
+                  want_arg: bool = True, arg: Optional[torch.Tensor] = None, stream=None):
+        """General AP.  Returns (fO, arg); arg is an int32 (n, F) tensor for max / min when
+        ``want_arg`` (allocated here unless given), else None."""
+        if F is None:
+            F = fV.shape[1] if fV is not None else fE.shape[1]
+        cols = self._edge_cols(fE, F)
+        if fO is None:
+            fO = torch.empty((self.n, F), dtype=torch.float32, device=self.device)
+        if reduce == DG_RED_SUM or not want_arg:
+            arg = None
+        elif arg is None:
+            arg = torch.empty((self.n, F), dtype=torch.int32, device=self.device)
+        _check(lib().dg_ap_fwd(self._h, _dev_ptr(fV, torch.float32, "fV"),
+                               _dev_ptr(fE, torch.float32, "fE"), cols, F, int(binary), int(reduce),
+                               _dev_ptr(fO, torch.float32, "fO"), _dev_ptr(arg, torch.int32, "arg"),
+                               _stream(stream)))
+        return fO, arg
+
+    def dg_ap_bwd(self, dO: torch.Tensor, fV: Optional[torch.Tensor], fE: Optional[torch.Tensor],
+                  binary: int, reduce: int, arg: Optional[torch.Tensor] = None, want_dV: bool = True,
+                  want_dE: bool = True, stream=None):
+        """Gradients of the general AP.  Returns (dV | None, dE | None)."""
+        F = dO.shape[1]
+        cols = self._edge_cols(fE, F)
+        dV = torch.empty((self.n, F), dtype=torch.float32, device=self.device) if want_dV else None
+        dE = None
+        if want_dE and binary != DG_BIN_COPY_LHS:
+            dE = torch.empty((self.nnz, cols), dtype=torch.float32, device=self.device)
+        _check(lib().dg_ap_bwd(self._h, _dev_ptr(dO, torch.float32, "dO"),
+                               _dev_ptr(fV, torch.float32, "fV"), _dev_ptr(fE, torch.float32, "fE"),
+                               cols, F, int(binary), int(reduce), _dev_ptr(arg, torch.int32, "arg"),
+                               _dev_ptr(dV, torch.float32, "dV"), _dev_ptr(dE, torch.float32, "dE"),
+                               _stream(stream)))
+        return dV, dE
+
+    def dg_aggregate_edge_grad(self, H: torch.Tensor, dOut: torch.Tensor, op: int,
+                               dW: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        F = H.shape[1]
+        if dOut.shape != H.shape:
+            raise ValueError("H and dOut must have the same shape")
+        if dW is None:
+            dW = torch.empty(self.nnz, dtype=torch.float32, device=self.device)
+        _check(lib().dg_aggregate_edge_grad(self._h, _dev_ptr(H, torch.float32, "H"),
+                                            _dev_ptr(dOut, torch.float32, "dOut"), F, int(op),
+                                            _dev_ptr(dW, torch.float32, "dW"), _stream(stream)))
+        return dW
 
     def dg_aggregate_host_workspace(self, F: int) -> int:
         return int(lib().dg_aggregate_host_workspace(self._h, int(F)))

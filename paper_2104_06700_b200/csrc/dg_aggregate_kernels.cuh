@@ -295,18 +295,25 @@ __device__ __forceinline__ void combine_groups(typename Vec<VEC>::T (&acc)[CPL])
   }
 }
 
-// A warp of a heavy segment moves its register sums into its shared-memory partial every
-// kHeavyFold batches, so that no fp32 chain is longer than 32 * kHeavyFold terms however long the
-// segment is: a segment of m entries is summed as chains of at most 512 terms, whose results form
-// a second chain of m / 4096 terms per warp, and the 8 warp partials are added last.  (One
-// register chain per warp, m / 8 terms, drifts past 1e-5 of the sum of magnitudes for same-sign
-// inputs once m reaches about 10^6.)
-constexpr int kHeavyFold = 16;
+// Graphs that hold a segment of kLongSegment entries or more run the kernels compiled with
+// FOLD: there a warp of a heavy segment moves its register sums into its shared-memory partial
+// every kLongFold batches, so that no fp32 chain is longer than 32 * kLongFold = 512 terms however
+// long the segment is (a segment of m entries is summed as chains of at most 512 terms, whose
+// results form a second chain of m / 4096 terms per warp, and the 8 warp partials are added last).
+// One register chain per warp, m / 8 terms, drifts past 1e-5 of the sum of magnitudes for
+// same-sign inputs once m reaches about 10^6; below kLongSegment it is at most 4096 terms long.
+// The fold is a second compilation of the kernels rather than a branch in one: in any of five
+// forms tried (a counter in the loop, a second loop for long segments, a shared-memory counter,
+// a function that is not inlined, a kernel of its own after the common one) it either changed the
+// register allocation of the common kernels (Reddit-like backward 17.8 -> 18.7 ms) or serialised
+// the long segments behind the rest (Papers-like backward 11.3 -> 16.0 ms at a tenth of the size).
+constexpr int kLongSegment = 1 << 15;
+constexpr int kLongFold = 16;
 
 // Block-per-row path for the heavy segments: block x of the first `heavy_blocks` blocks takes
 // entries x, x + heavy_blocks, ... of the heavy list; its 8 warps sum interleaved 32-edge
 // batches and the partial sums are combined in shared memory in warp order.
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool SELF>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool SELF, bool FOLD>
 __device__ __forceinline__ void heavy_rows(const ApArgs& a, const SelfArgs sa,
                                            const int heavy_blocks,
                                            float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
@@ -338,22 +345,11 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const SelfArgs sa,
     V acc[CPL];
 #pragma unroll
     for (int c = 0; c < CPL; ++c) zero(acc[c]);
-    if (lane < G) {
+    if (FOLD && lane < G) {
 #pragma unroll
       for (int c = 0; c < CPL; ++c)
         if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
     }
-    // adds the warp's register sums to its partial in shared memory and starts them afresh
-    auto fold = [&]() {
-      combine_groups<VEC, G, CPL>(acc);
-      if (lane < G) {
-#pragma unroll
-        for (int c = 0; c < CPL; ++c)
-          if (cok[c]) add_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
-      }
-#pragma unroll
-      for (int c = 0; c < CPL; ++c) zero(acc[c]);
-    };
     // warp w sums batches w, w+8, ... of the segment
     int32_t cur_u, nxt_u;
     float cur_s, nxt_s;
@@ -365,16 +361,31 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const SelfArgs sa,
       if (more) load_batch<SCALED>(a, (int64_t)b + kBlock, hi, lane, nxt_u, nxt_s);
       add_edges<E, VEC, G, CPL, SCALED, SEG>(xrow, row_bytes, cur_u, cur_s, 0, min(hi - b, 32), grp, acc,
                                      stage);
-      if (!more) break;
-      if (++since_fold == kHeavyFold) {
-        fold();
+      if (FOLD && (++since_fold == kLongFold || !more)) {
+        // the register sums join the warp's partial in shared memory and start afresh
         since_fold = 0;
+        combine_groups<VEC, G, CPL>(acc);
+        if (lane < G) {
+#pragma unroll
+          for (int c = 0; c < CPL; ++c)
+            if (cok[c]) add_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
+        }
+#pragma unroll
+        for (int c = 0; c < CPL; ++c) zero(acc[c]);
       }
+      if (!more) break;
       b += kBlock;
       cur_u = nxt_u;
       cur_s = nxt_s;
     }
-    fold();
+    if (!FOLD) {
+      combine_groups<VEC, G, CPL>(acc);
+      if (lane < G) {
+#pragma unroll
+        for (int c = 0; c < CPL; ++c)
+          if (cok[c]) st_smem(&part[warp][(c0 + c * G) * VEC], acc[c]);
+      }
+    }
     __syncthreads();
     float* orow = a.Y + (size_t)r * (size_t)a.F + f0;
     if constexpr (SELF) {
@@ -409,7 +420,7 @@ __device__ __forceinline__ void heavy_rows(const ApArgs& a, const SelfArgs sa,
 // first, so the long segments start early); in the remaining blocks every warp owns
 // rows_per_warp consecutive light segments and streams their indices as one run of 32-edge
 // batches, the next batch always in flight while the current one is summed.
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool SELF>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool SELF, bool FOLD>
 __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
                                         const int heavy_blocks,
                                         float (&part)[kWarpsPerBlock][32 * CPL * VEC]) {
@@ -596,13 +607,13 @@ __device__ __forceinline__ void ap_body(const ApArgs& a, const SelfArgs sa,
     return;
   }
 
-  heavy_rows<E, VEC, G, CPL, SCALED, SEG, SELF>(a, sa, heavy_blocks, part);
+  heavy_rows<E, VEC, G, CPL, SCALED, SEG, SELF, FOLD>(a, sa, heavy_blocks, part);
 }
 
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool FOLD>
 __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int heavy_blocks) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<E, VEC, G, CPL, SCALED, SEG, false>(a, SelfArgs{}, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG, false, FOLD>(a, SelfArgs{}, heavy_blocks, part);
 }
 
 // The same kernel compiled for six resident blocks per SM (at most 40 registers).  The scaled
@@ -611,25 +622,25 @@ __global__ void __launch_bounds__(kBlock) ap_kernel(const ApArgs a, const int he
 // higher occupancy wins for them (Reddit-like backward 22.0 ms uncapped, 19.2 ms at five
 // blocks, 18.3 ms at six, 20.0 ms at seven or eight; Products-like backward 7.0 -> 5.9 ms),
 // while a cap slows the unscaled variants down.
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool FOLD>
 __global__ void __launch_bounds__(kBlock, 6) ap_kernel_r40(const ApArgs a, const int heavy_blocks) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<E, VEC, G, CPL, SCALED, SEG, false>(a, SelfArgs{}, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG, false, FOLD>(a, SelfArgs{}, heavy_blocks, part);
 }
 
 // Both again for graphs with implicit self loops: every row also sums its own input row.
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool FOLD>
 __global__ void __launch_bounds__(kBlock) ap_kernel_self(const ApArgs a, const int heavy_blocks,
                                                          const SelfArgs sa) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<E, VEC, G, CPL, SCALED, SEG, true>(a, sa, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG, true, FOLD>(a, sa, heavy_blocks, part);
 }
 
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG>
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SEG, bool FOLD>
 __global__ void __launch_bounds__(kBlock, 6) ap_kernel_self_r40(const ApArgs a, const int heavy_blocks,
                                                                 const SelfArgs sa) {
   __shared__ float part[kWarpsPerBlock][32 * CPL * VEC];
-  ap_body<E, VEC, G, CPL, SCALED, SEG, true>(a, sa, heavy_blocks, part);
+  ap_body<E, VEC, G, CPL, SCALED, SEG, true, FOLD>(a, sa, heavy_blocks, part);
 }
 
 // Blocks that walk the heavy list: as many as the device keeps resident, so that the heavy
@@ -644,21 +655,21 @@ int heavy_block_count(const Graph* g, K kernel, size_t smem) {
   return g->sm_count * (per_sm < 1 ? 1 : per_sm);
 }
 
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SELF>
-dg_status_t launch_pair(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
-                        cudaStream_t s) {
-  if (a.n == 0) return DG_OK;
+// FOLD: the graph may hold segments of kLongSegment entries or more in this direction.
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SELF, bool FOLD>
+dg_status_t launch_variant(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
+                           cudaStream_t s) {
   constexpr bool kCapped = SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16;
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
   const int64_t light_blocks = (a.n + rows_per_block - 1) / rows_per_block;
   if constexpr (SELF) {
     void (*kernel)(const ApArgs, const int, const SelfArgs);
     if constexpr (kCapped) {
-      kernel = a.seg_lo ? ap_kernel_self_r40<E, VEC, G, CPL, SCALED, true>
-                        : ap_kernel_self_r40<E, VEC, G, CPL, SCALED, false>;
+      kernel = a.seg_lo ? ap_kernel_self_r40<E, VEC, G, CPL, SCALED, true, FOLD>
+                        : ap_kernel_self_r40<E, VEC, G, CPL, SCALED, false, FOLD>;
     } else {
-      kernel = a.seg_lo ? ap_kernel_self<E, VEC, G, CPL, SCALED, true>
-                        : ap_kernel_self<E, VEC, G, CPL, SCALED, false>;
+      kernel = a.seg_lo ? ap_kernel_self<E, VEC, G, CPL, SCALED, true, FOLD>
+                        : ap_kernel_self<E, VEC, G, CPL, SCALED, false, FOLD>;
     }
     const int heavy_blocks = heavy_block_count(g, kernel, 0);
     dim3 grid((unsigned)(heavy_blocks + light_blocks), (unsigned)slices);
@@ -666,11 +677,11 @@ dg_status_t launch_pair(const Graph* g, const ApArgs& a, const SelfArgs& sa, int
   } else {
     void (*kernel)(const ApArgs, const int);
     if constexpr (kCapped) {
-      kernel = a.seg_lo ? ap_kernel_r40<E, VEC, G, CPL, SCALED, true>
-                        : ap_kernel_r40<E, VEC, G, CPL, SCALED, false>;
+      kernel = a.seg_lo ? ap_kernel_r40<E, VEC, G, CPL, SCALED, true, FOLD>
+                        : ap_kernel_r40<E, VEC, G, CPL, SCALED, false, FOLD>;
     } else {
-      kernel = a.seg_lo ? ap_kernel<E, VEC, G, CPL, SCALED, true>
-                        : ap_kernel<E, VEC, G, CPL, SCALED, false>;
+      kernel = a.seg_lo ? ap_kernel<E, VEC, G, CPL, SCALED, true, FOLD>
+                        : ap_kernel<E, VEC, G, CPL, SCALED, false, FOLD>;
     }
     const int heavy_blocks = heavy_block_count(g, kernel, 0);
     dim3 grid((unsigned)(heavy_blocks + light_blocks), (unsigned)slices);
@@ -679,6 +690,14 @@ dg_status_t launch_pair(const Graph* g, const ApArgs& a, const SelfArgs& sa, int
   DG_CUDA(cudaGetLastError());
   count_launches(1);
   return DG_OK;
+}
+
+template <typename E, int VEC, int G, int CPL, bool SCALED, bool SELF>
+dg_status_t launch_pair(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
+                        cudaStream_t s) {
+  if (a.n == 0) return DG_OK;
+  return a.long_segments ? launch_variant<E, VEC, G, CPL, SCALED, SELF, true>(g, a, sa, slices, s)
+                         : launch_variant<E, VEC, G, CPL, SCALED, SELF, false>(g, a, sa, slices, s);
 }
 
 template <typename E, int VEC, bool SCALED, bool SELF>

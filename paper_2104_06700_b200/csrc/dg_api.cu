@@ -45,6 +45,11 @@ static dg_status_t free_owned(Graph* g) {
   if (g->counters) cudaFree(g->counters);
   if (g->split_csr) cudaFree(g->split_csr);
   g->split_csr = nullptr;
+  if (g->long_cols_host) cudaFreeHost(g->long_cols_host);
+  g->long_cols_host = nullptr;
+  if (g->long_cols_ready) cudaEventDestroy(g->long_cols_ready);
+  g->long_cols_ready = nullptr;
+
   for (size_t i = 0; i < g->aux_event_count; ++i) cudaEventDestroy(g->aux_events[i]);
   free(g->aux_events);
   g->aux_events = nullptr;
@@ -69,6 +74,36 @@ static dg_status_t refresh_heavy(Graph* g, bool csr, bool csc, cudaStream_t s) {
                                           g->heavy_cap, g->counters + 1, s))
       return st;
   return DG_OK;
+}
+
+// Index of the length class of the heavy-list builder at which segments of 2^15 entries start;
+// after the list is filled, counter [class] holds the number of segments in that class or above.
+constexpr int kLongClass = 30;
+
+// Heavy columns of a fresh CSC, and the number of long ones sent to the host behind them (read
+// by the first backward pass that finds the copy finished; until then the columns count as long).
+dg_status_t finish_transpose(Graph* g, cudaStream_t s) {
+  if (dg_status_t st = refresh_heavy(g, false, true, s)) return st;
+  g->long_cols = -1;
+  DG_CUDA(cudaMemcpyAsync(g->long_cols_host, g->heavy_cols + g->heavy_cap + kLongClass,
+                          sizeof(int32_t), cudaMemcpyDeviceToHost, s));
+  DG_CUDA(cudaEventRecord(g->long_cols_ready, s));
+  return DG_OK;
+}
+
+// Synchronous: the heavy rows have just been (re)built on the default stream.
+static dg_status_t count_long_rows(Graph* g) {
+  int32_t longs = 0;
+  DG_CUDA(cudaMemcpy(&longs, g->heavy_rows + g->heavy_cap + kLongClass, sizeof(longs),
+                     cudaMemcpyDeviceToHost));
+  g->long_rows = longs > 0 ? 1 : 0;
+  return DG_OK;
+}
+
+static int long_columns(Graph* g) {
+  if (g->long_cols < 0 && cudaEventQuery(g->long_cols_ready) == cudaSuccess)
+    g->long_cols = *g->long_cols_host > 0 ? 1 : 0;
+  return g->long_cols != 0;
 }
 
 // rows_per_block is rounded up to a whole number of rows per warp (8 warps per block).  0 picks
@@ -127,6 +162,7 @@ static dg_status_t run_forward(Graph* g, const void* H, bool bf16, int32_t F, dg
   a.mean_rows = op == DG_OP_MEAN;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
+  a.long_segments = g->long_rows;
   const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
   return aggregate_run(g, a, sa, g->split_csr, (cudaStream_t)stream);
 }
@@ -157,6 +193,7 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   a.mean_rows = 0;
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
+  a.long_segments = long_columns(g);
   const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
   return aggregate_run(g, a, sa, g->split_csc, (cudaStream_t)stream);
 }
@@ -212,6 +249,8 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (e == cudaSuccess) e = cudaMalloc(&g->heavy_rows, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->heavy_cols, (size_t)(g->heavy_cap + kHeavyListExtra) * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&g->counters, 4 * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaHostAlloc(&g->long_cols_host, sizeof(int32_t), cudaHostAllocDefault);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g->long_cols_ready, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaMemset(g->counters, 0, 4 * sizeof(int32_t));
   if (e == cudaSuccess && wants_split(n, nnz))
     e = cudaMalloc(&g->split_csr, (size_t)(kFineBlocks + 1) * (size_t)n * sizeof(int32_t));
@@ -225,6 +264,7 @@ dg_status_t dg_graph_create(int64_t n, int64_t nnz, const int64_t* rowptr,
   if (st == DG_OK) st = refresh_heavy(g, true, false, 0);
   if (st == DG_OK && g->split_csr)
     st = build_split(rowptr, colidx, n, g->fine_rows, g->split_csr, g->counters + 3, 0);
+  if (st == DG_OK) st = count_long_rows(g);
   if (st == DG_OK) {
     int32_t unsorted = 0;
     e = cudaMemcpy(&unsorted, g->counters + 3, sizeof(unsorted), cudaMemcpyDeviceToHost);
@@ -278,7 +318,14 @@ dg_status_t dg_graph_transpose(dg_graph_t g, void* csc_storage, size_t csc_bytes
   g->transposed = false;
   if (dg_status_t st = transpose_run(g, csc_storage, scratch, (cudaStream_t)stream)) return st;
   g->transposed = true;
-  return refresh_heavy(g, false, true, (cudaStream_t)stream);
+  return finish_transpose(g, (cudaStream_t)stream);
+}
+
+dg_status_t dg_graph_update_weights(dg_graph_t g, void* stream) {
+  if (!g) return invalid("graph handle is NULL");
+  if (!g->edge_w) return invalid("the graph has no edge weights");
+  if (!g->transposed) return DG_OK;  // the CSR is read in place: nothing to refresh
+  return refresh_csc_weights(g, (cudaStream_t)stream);
 }
 
 dg_status_t dg_graph_get_csc(dg_graph_t g, const int64_t** colptr, const int32_t** rowidx_T,
@@ -428,7 +475,10 @@ dg_status_t dg_graph_set_param(dg_graph_t g, const char* name, int64_t value) {
     // the lists may be in use, or being built, on any stream: wait for the device on both sides
     DG_CUDA(cudaDeviceSynchronize());
     g->heavy_threshold = value;
-    if (dg_status_t st = refresh_heavy(g, true, true, 0)) return st;
+    if (dg_status_t st = refresh_heavy(g, true, false, 0)) return st;
+    if (dg_status_t st = count_long_rows(g)) return st;
+    if (g->transposed)
+      if (dg_status_t st = finish_transpose(g, 0)) return st;
     DG_CUDA(cudaDeviceSynchronize());
     return DG_OK;
   }

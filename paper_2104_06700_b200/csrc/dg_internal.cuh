@@ -34,6 +34,14 @@ struct dg_graph {
   cudaEvent_t* aux_events = nullptr;  // malloc'ed pool, aux_event_count entries
   size_t aux_event_count = 0;
 
+  // Whether a CSR row / CSC column of 2^15 entries or more exists (1), does not (0), or is not
+  // known yet (-1: the count of the last transposition is still on its way to the host).  Such
+  // graphs run the kernels compiled with the two-level sum of the block-per-row path.
+  int long_rows = 1;
+  int long_cols = -1;
+  int32_t* long_cols_host = nullptr;     // pinned; written by a copy enqueued after a transposition
+  cudaEvent_t long_cols_ready = nullptr; // recorded behind that copy
+
   bool transposed = false;
   const int64_t* colptr = nullptr;
   const int32_t* rowidx_T = nullptr;
@@ -42,6 +50,10 @@ struct dg_graph {
   const float* mean_scale_T = nullptr;  // w_T[q] / (deg(rowidx_T[q]) + self_loops): edge factor of the mean's backward
   int64_t self_loops = 0;        // 1: every vertex is its own in-neighbour with weight 1
   int64_t self_loops_in_csc = 0; // value mean_scale_T was built with
+
+  // set on a handle made by dg_graph_reorder: arrays inside the caller's reorder storage
+  const int32_t* new_of_old = nullptr;   // n: new id of every old vertex
+  const int32_t* reorder_pos = nullptr;  // nnz: old CSR position of every new position
 
   int device = 0;
   int sm_count = 148;
@@ -84,6 +96,7 @@ struct ApArgs {
   const int32_t* seg_lo;      // source-blocked pass: first and one-past-last position of every
   const int32_t* seg_hi;      //   segment's piece (n entries each); nullptr = whole segments
   int32_t accumulate;         // source-blocked pass after the first: add to what Y holds
+  int32_t long_segments;      // host side only: a segment of 2^15 entries or more may exist
 };
 
 // Implicit self loops (every vertex its own neighbour with weight 1): row r also receives
@@ -127,6 +140,20 @@ dg_status_t build_split(const int64_t* ptr, const int32_t* idx, int64_t n, int64
 void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
                      size_t* scratch_bytes);
 dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s);
+dg_status_t refresh_csc_weights(Graph* g, cudaStream_t s);
+// dg_api.cu: what follows every transposition (heavy columns, the long-column count on its way)
+dg_status_t finish_transpose(Graph* g, cudaStream_t s);
+// the stable radix sort behind it, for other pre-processing steps (see dg_transpose.cu)
+int sort_passes(int64_t key_range);
+void sort_scratch_sizes(int64_t count, size_t* hist_bytes, size_t* sums_bytes);
+dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count, int passes,
+                       uint32_t* const keys_buf[2], uint32_t* vals_final, uint32_t* vals_tmp,
+                       uint32_t* hist, uint32_t* sums, const uint32_t** sorted_keys,
+                       cudaStream_t s);
+dg_status_t pointers_from_sorted_keys(const uint32_t* sorted, int64_t count, int64_t n,
+                                      int64_t* ptr, cudaStream_t s);
+dg_status_t expand_rows(const int64_t* rowptr, int64_t n, int64_t nnz, const int32_t* map,
+                        uint32_t* out, cudaStream_t s);
 
 // dg_aggregate.cu
 dg_status_t aggregate_run(const Graph* g, const ApArgs& a, const SelfArgs& sa, const int32_t* split,

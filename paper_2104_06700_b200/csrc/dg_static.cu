@@ -81,6 +81,5 @@ extern "C" dg_status_t dg_graph_transpose_static(dg_graph_t g, void* csc_storage
   g->transposed = false;
   if (dg_status_t st = dg::transpose_run(g, csc_storage, scratch, s)) return st;
   g->transposed = true;
-  return dg::build_heavy_list(g->colptr, g->n, g->heavy_threshold, g->heavy_cols, g->heavy_cap,
-                              g->counters + 1, s);
+  return dg::finish_transpose(g, s);
 }

@@ -338,6 +338,42 @@ __global__ void row_info_kernel(const int64_t* __restrict__ rowptr, int self, in
   }
 }
 
+// The same walk with another payload: out[k] = map[r] (or r) for the row r that holds position k.
+__global__ void expand_rows_kernel(const int64_t* __restrict__ rowptr, int64_t n, int64_t nnz,
+                                   const int32_t* __restrict__ map, uint32_t* __restrict__ out) {
+  const int64_t k0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kRowItems;
+  if (k0 >= nnz) return;
+  int64_t lo = 0, hi = n;  // invariant: rowptr[lo] <= k0 < rowptr[hi]
+  while (hi - lo > 1) {
+    const int64_t mid = (lo + hi) >> 1;
+    if (__ldg(rowptr + mid) <= k0) lo = mid; else hi = mid;
+  }
+  int64_t r = lo;
+  int64_t r_end = __ldg(rowptr + r + 1);
+  uint32_t payload = map ? (uint32_t)__ldg(map + r) : (uint32_t)r;
+#pragma unroll 1
+  for (int i = 0; i < kRowItems; ++i) {
+    const int64_t k = k0 + i;
+    if (k >= nnz) break;
+    if (k >= r_end) {
+      int64_t step = 1, lo2 = r, hi2 = r + 1;
+      while (hi2 < n && __ldg(rowptr + hi2) <= k) {
+        lo2 = hi2;
+        step <<= 1;
+        hi2 = hi2 + step < n ? hi2 + step : n;
+      }
+      while (hi2 - lo2 > 1) {
+        const int64_t mid = (lo2 + hi2) >> 1;
+        if (__ldg(rowptr + mid) <= k) lo2 = mid; else hi2 = mid;
+      }
+      r = lo2;
+      r_end = __ldg(rowptr + r + 1);
+      payload = map ? (uint32_t)__ldg(map + r) : (uint32_t)r;
+    }
+    out[k] = payload;
+  }
+}
+
 // rowidx_T[q] = row of perm[q];  w_T[q] = edge_w[perm[q]];  mean_scale_T[q] = w_T[q] (1 if
 // unweighted) / (deg(row) + self), the factor of edge q in the backward pass of the mean, so that
 // the backward kernel streams it instead of gathering 1/deg.  One 8-byte gather per edge.
@@ -357,6 +393,21 @@ __global__ void gather_rows_and_weights(const uint32_t* __restrict__ perm, int64
     w_T[q] = w;
   }
   mean_scale_T[q] = w * __uint_as_float(info.y);
+}
+
+// After the caller changed edge_w in place (learnable edge weights): the two weight arrays of the
+// CSC again, from perm.  The in-degree comes from the CSR row pointer.
+__global__ void regather_weights_kernel(const uint32_t* __restrict__ perm, int64_t nnz,
+                                        const float* __restrict__ edge_w,
+                                        const int32_t* __restrict__ rowidx_T,
+                                        const int64_t* __restrict__ rowptr, int self,
+                                        float* __restrict__ w_T, float* __restrict__ mean_scale_T) {
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= nnz) return;
+  const float w = edge_w[perm[q]];
+  const int64_t v = rowidx_T[q];
+  w_T[q] = w;
+  mean_scale_T[q] = w * (1.0f / (float)(__ldg(rowptr + v + 1) - __ldg(rowptr + v) + self));
 }
 
 inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
@@ -381,9 +432,7 @@ Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
   L.mscale_off = o; o += align256((size_t)nnz * 4);
   L.split_off = o;  o += wants_split(n, nnz) ? align256((size_t)(kFineBlocks + 1) * n * 4) : 0;
   L.csc_bytes = o > 0 ? o : 256;
-  int bits = 1;
-  while (bits < 31 && ((int64_t)1 << bits) < n) ++bits;
-  L.passes = (bits + kRadixBits - 1) / kRadixBits;
+  L.passes = sort_passes(n);
   L.tiles = (nnz + kTile - 1) / kTile;
   L.hist_len = L.tiles * kRadix;
   L.chunks = (L.hist_len + kScanChunk - 1) / kScanChunk;
@@ -399,11 +448,92 @@ Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
 
 }  // namespace
 
+int sort_passes(int64_t key_range) {
+  int bits = 1;
+  while (bits < 31 && ((int64_t)1 << bits) < key_range) ++bits;
+  return (bits + kRadixBits - 1) / kRadixBits;
+}
+
+void sort_scratch_sizes(int64_t count, size_t* hist_bytes, size_t* sums_bytes) {
+  const int64_t tiles = (count + kTile - 1) / kTile;
+  const int64_t hist_len = tiles * kRadix;
+  const int64_t chunks = (hist_len + kScanChunk - 1) / kScanChunk;
+  *hist_bytes = align256((size_t)(hist_len > 0 ? hist_len : 1) * 4);
+  *sums_bytes = align256((size_t)(chunks > 0 ? chunks : 1) * 4);
+}
+
+// Stable LSD radix sort of `count` (key, value) pairs over `passes` digits.  vals_in == nullptr
+// means "the value of key i is i".  keys_in is only read; the sorted keys end in one of keys_buf
+// (reported through *sorted_keys; keys_in may be keys_buf[1], which is first written by the second
+// pass), the sorted values in vals_final (vals_tmp is the other buffer of the ping-pong).
+dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count, int passes,
+                       uint32_t* const keys_buf[2], uint32_t* vals_final, uint32_t* vals_tmp,
+                       uint32_t* hist, uint32_t* sums, const uint32_t** sorted_keys,
+                       cudaStream_t s) {
+  const int64_t tiles = (count + kTile - 1) / kTile;
+  const int64_t hist_len = tiles * kRadix;
+  const int64_t chunks = (hist_len + kScanChunk - 1) / kScanChunk;
+  for (int p = 0; p < passes; ++p) {
+    const int shift = p * kRadixBits;
+    // value buffers alternate so that the last pass lands in vals_final
+    uint32_t* vals_out = ((passes - 1 - p) % 2 == 0) ? vals_final : vals_tmp;
+    uint32_t* keys_out = keys_buf[p % 2];
+    digit_histogram<<<(unsigned)tiles, kSortBlock, 0, s>>>(keys_in, count, shift, tiles,
+                                                           aligned16(keys_in), hist);
+    DG_CUDA(cudaGetLastError());
+    scan_reduce<<<(unsigned)chunks, kScanBlock, 0, s>>>(hist, hist_len, sums);
+    DG_CUDA(cudaGetLastError());
+    scan_spine<<<1, kScanBlock, 0, s>>>(sums, chunks);
+    DG_CUDA(cudaGetLastError());
+    scan_apply<<<(unsigned)chunks, kScanBlock, 0, s>>>(hist, hist_len, sums);
+    DG_CUDA(cudaGetLastError());
+    digit_scatter<<<(unsigned)tiles, kSortBlock, 0, s>>>(keys_in, vals_in, count, shift, tiles,
+                                                         hist, keys_out, vals_out);
+    DG_CUDA(cudaGetLastError());
+    count_launches(5);
+    keys_in = keys_out;
+    vals_in = vals_out;
+  }
+  *sorted_keys = keys_in;
+  return DG_OK;
+}
+
+// ptr[u] = first position whose sorted key is >= u, for u = 0..n (ptr[n] = count)
+dg_status_t pointers_from_sorted_keys(const uint32_t* sorted, int64_t count, int64_t n,
+                                      int64_t* ptr, cudaStream_t s) {
+  const unsigned blocks = (unsigned)(((count + kColptrItems) / kColptrItems + 255) / 256);
+  colptr_from_sorted_keys<<<blocks, 256, 0, s>>>(sorted, count, n, aligned16(sorted), ptr);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
+}
+
+// out[k] = map[r] (r itself when map is nullptr) for the CSR row r that contains position k
+dg_status_t expand_rows(const int64_t* rowptr, int64_t n, int64_t nnz, const int32_t* map,
+                        uint32_t* out, cudaStream_t s) {
+  if (nnz == 0) return DG_OK;
+  const unsigned blocks = (unsigned)(((nnz + kRowItems - 1) / kRowItems + 255) / 256);
+  expand_rows_kernel<<<blocks, 256, 0, s>>>(rowptr, n, nnz, map, out);
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
+}
+
 void transpose_sizes(int64_t n, int64_t nnz, bool weighted, size_t* csc_bytes,
                      size_t* scratch_bytes) {
   const Layout L = make_layout(n, nnz, weighted);
   *csc_bytes = L.csc_bytes;
   *scratch_bytes = L.scratch_bytes;
+}
+
+dg_status_t refresh_csc_weights(Graph* g, cudaStream_t s) {
+  if (g->nnz == 0 || !g->edge_w) return DG_OK;
+  regather_weights_kernel<<<(unsigned)((g->nnz + 255) / 256), 256, 0, s>>>(
+      reinterpret_cast<const uint32_t*>(g->perm), g->nnz, g->edge_w, g->rowidx_T, g->rowptr,
+      g->self_loops_in_csc ? 1 : 0, const_cast<float*>(g->w_T), const_cast<float*>(g->mean_scale_T));
+  DG_CUDA(cudaGetLastError());
+  count_launches(1);
+  return DG_OK;
 }
 
 dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
@@ -426,32 +556,11 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
   if (nnz == 0) {
     DG_CUDA(cudaMemsetAsync(colptr, 0, (size_t)(n + 1) * 8, s));
   } else {
-    const uint32_t* keys_in = reinterpret_cast<const uint32_t*>(g->colidx);
-    const uint32_t* vals_in = nullptr;
-    for (int p = 0; p < L.passes; ++p) {
-      const int shift = p * kRadixBits;
-      // value buffers alternate so that the last pass lands in perm
-      uint32_t* vals_out = ((L.passes - 1 - p) % 2 == 0) ? perm : vals_tmp;
-      uint32_t* keys_out = keys_buf[p % 2];
-      digit_histogram<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, nnz, shift, L.tiles,
-                                                               aligned16(keys_in), hist);
-      DG_CUDA(cudaGetLastError());
-      scan_reduce<<<(unsigned)L.chunks, kScanBlock, 0, s>>>(hist, L.hist_len, sums);
-      DG_CUDA(cudaGetLastError());
-      scan_spine<<<1, kScanBlock, 0, s>>>(sums, L.chunks);
-      DG_CUDA(cudaGetLastError());
-      scan_apply<<<(unsigned)L.chunks, kScanBlock, 0, s>>>(hist, L.hist_len, sums);
-      DG_CUDA(cudaGetLastError());
-      digit_scatter<<<(unsigned)L.tiles, kSortBlock, 0, s>>>(keys_in, vals_in, nnz, shift,
-                                                            L.tiles, hist, keys_out, vals_out);
-      DG_CUDA(cudaGetLastError());
-      count_launches(5);
-      keys_in = keys_out;
-      vals_in = vals_out;
-    }
-    const unsigned b1 = (unsigned)(((nnz + kColptrItems) / kColptrItems + 255) / 256);
-    colptr_from_sorted_keys<<<b1, 256, 0, s>>>(keys_in, nnz, n, aligned16(keys_in), colptr);
-    DG_CUDA(cudaGetLastError());
+    const uint32_t* keys_in = nullptr;
+    if (dg_status_t st = sort_pairs(reinterpret_cast<const uint32_t*>(g->colidx), nullptr, nnz,
+                                    L.passes, keys_buf, perm, vals_tmp, hist, sums, &keys_in, s))
+      return st;
+    if (dg_status_t st = pointers_from_sorted_keys(keys_in, nnz, n, colptr, s)) return st;
     const unsigned b2 = (unsigned)((nnz + 255) / 256);
     // colptr has been derived from the sorted keys (stream order), so both key buffers, which
     // are adjacent in the scratch, are free: they hold the nnz (row, 1/deg) pairs
@@ -462,7 +571,7 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
     gather_rows_and_weights<<<b2, 256, 0, s>>>(perm, nnz, row_info, g->edge_w, rowidx_T, w_T,
                                                mean_scale_T);
     DG_CUDA(cudaGetLastError());
-    count_launches(3);
+    count_launches(2);
   }
   g->colptr = colptr;
   g->rowidx_T = rowidx_T;

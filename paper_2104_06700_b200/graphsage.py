@@ -31,8 +31,13 @@ class _Aggregate(torch.autograd.Function):
 
     @staticmethod
     def forward(ctx, H: torch.Tensor, graph: "binding.Graph", op: int, bf16: bool,
-                row_scale) -> torch.Tensor:
+                row_scale, edge_w=None) -> torch.Tensor:
         ctx.graph, ctx.op, ctx.bf16, ctx.row_scale = graph, op, bf16, row_scale
+        ctx.want_dw = edge_w is not None and edge_w.requires_grad
+        if ctx.want_dw:
+            if edge_w.data_ptr() != graph.edge_w.data_ptr():
+                raise ValueError("edge_w must be the tensor the graph handle was created with")
+            ctx.save_for_backward(H)
         if bf16:
             return graph.dg_aggregate_fwd_bf16(H.contiguous().to(torch.bfloat16), op)
         return graph.dg_aggregate_fwd(H.contiguous(), op)
@@ -40,6 +45,7 @@ class _Aggregate(torch.autograd.Function):
     @staticmethod
     def backward(ctx, dOut: torch.Tensor):
         dH = None
+        upstream = dOut
         if ctx.needs_input_grad[0]:
             op = ctx.op
             if ctx.row_scale is not None:
@@ -49,13 +55,22 @@ class _Aggregate(torch.autograd.Function):
                 dH = ctx.graph.dg_aggregate_bwd_bf16(dOut.contiguous().to(torch.bfloat16), op)
             else:
                 dH = ctx.graph.dg_aggregate_bwd(dOut.contiguous(), op)
-        return dH, None, None, None, None
+        dW = None
+        if ctx.want_dw:     # message passing onto the edges: one dot product per edge
+            (H,) = ctx.saved_tensors
+            dW = ctx.graph.dg_aggregate_edge_grad(H.contiguous(), upstream.contiguous(), ctx.op)
+        return dH, None, None, None, None, dW
 
 
 def aggregate(graph: "binding.Graph", H: torch.Tensor, op: int = binding.DG_OP_SUM,
-              bf16: bool = False, row_scale=None) -> torch.Tensor:
-    """Differentiable aggregation primitive (the graph must have been transposed)."""
-    return _Aggregate.apply(H, graph, op, bf16, row_scale)
+              bf16: bool = False, row_scale=None, edge_w=None) -> torch.Tensor:
+    """Differentiable aggregation primitive (the graph must have been transposed).
+
+    ``edge_w``: pass the weight tensor the handle was created with to get its gradient too
+    (learnable edge weights).  The handle reads that tensor in place; after an optimiser step
+    on it call ``graph.dg_graph_update_weights()`` so that the CSC used by the backward pass
+    carries the new values."""
+    return _Aggregate.apply(H, graph, op, bf16, row_scale, edge_w)
 
 
 class GraphSAGE(torch.nn.Module):

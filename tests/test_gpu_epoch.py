@@ -108,3 +108,42 @@ def test_fused_aggregator_needs_the_matching_handle():
     g.dg_graph_set_param("self_loops", 1)
     with pytest.raises(ValueError):
         graphsage.GraphSAGE(g, [8, 4])
+
+
+@pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
+def test_learnable_edge_weights_gradient_and_refresh(op):
+    """The autograd wrapper returns the gradient with respect to the edge weights (one dot product
+    per edge, dg_aggregate_edge_grad) next to the one for the features; after an in-place update of
+    the weights dg_graph_update_weights brings the CSC of the backward pass up to date.  Reference:
+    index_add_ with autograd in fp64."""
+    sg = synth.make("tiny")
+    rowptr, colidx = sg.rowptr.to(DEV), sg.colidx.to(DEV)
+    w = sg.edge_w.to(DEV).clone().requires_grad_(True)
+    g = binding.dg_graph_create(sg.n, sg.nnz, rowptr, colidx, w.detach())
+    assert w.data_ptr() == g.edge_w.data_ptr()
+    g.dg_graph_transpose()
+    F = 48
+    rows = torch.repeat_interleave(torch.arange(sg.n, device=DEV), rowptr[1:] - rowptr[:-1])
+    deg = (rowptr[1:] - rowptr[:-1]).double().clamp(min=1).unsqueeze(1)
+
+    def reference(H, wt):
+        out = torch.zeros((sg.n, F), dtype=torch.float64, device=DEV)
+        out.index_add_(0, rows, H.double()[colidx.long()] * wt.double().unsqueeze(1))
+        return out / deg if op == binding.DG_OP_MEAN else out
+
+    for step in range(2):
+        H = synth.features(sg.n, F, 70 + step, DEV).requires_grad_(True)
+        G = synth.features(sg.n, F, 80 + step, DEV)
+        out = graphsage.aggregate(g, H, op, edge_w=w)
+        (out * G).sum().backward()
+        Hr = H.detach().clone().requires_grad_(True)
+        wr = w.detach().clone().requires_grad_(True)
+        (reference(Hr, wr) * G.double()).sum().backward()
+        assert torch.allclose(out.detach().double(), reference(H.detach(), w.detach()),
+                              rtol=1e-4, atol=1e-4)
+        assert torch.allclose(H.grad.double(), Hr.grad.double(), rtol=1e-4, atol=1e-4)
+        assert torch.allclose(w.grad.double(), wr.grad.double(), rtol=1e-4, atol=1e-3)
+        with torch.no_grad():                       # an optimiser step on the weights, in place
+            w -= 0.05 * w.grad
+            w.grad = None
+        g.dg_graph_update_weights()

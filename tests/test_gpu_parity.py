@@ -291,6 +291,25 @@ def test_probe_gather_sums_the_rows_it_names():
     assert torch.allclose(got.double(), want, rtol=1e-4, atol=1e-3)
 
 
+@pytest.mark.parametrize("remote", [False, True])
+@pytest.mark.parametrize("rf", [8, 32, 128])
+def test_probe_gather_smem_sums_the_rows_it_names(rf, remote):
+    """Row r of the stage holds the value r, so a warp's sum over its 4096 gathers is the sum of
+    its indices (exact in fp32 at these sizes), from its own or its cluster partner's stage."""
+    stage_rows, count = 300, 3 * 4096 + 1000
+    idx = torch.randint(0, stage_rows, (count,), device=DEV, dtype=torch.int32)
+    warps = (count + 4095) // 4096
+    sink = torch.zeros((warps + 32) * 128, device=DEV)
+    binding.dg_probe_gather_smem(rf, stage_rows, idx, sink, remote)
+    torch.cuda.synchronize()
+    groups = 128 // rf
+    got = sink[:warps * 128].view(warps, groups, rf).sum(1)
+    want = torch.stack([idx[w * 4096:(w + 1) * 4096].double().sum().expand(rf) for w in range(warps)])
+    assert torch.equal(got.double(), want)
+    with pytest.raises(binding.DgError):
+        binding.dg_probe_gather_smem(128, 1000, idx, sink, remote)      # 512 KB stage
+
+
 # ------------------------------------------------------------------ errors never trap
 def test_error_statuses(tiny):
     g = make_graph(tiny)
