@@ -44,12 +44,12 @@ METRIC = "ap_fwd_bwd_edge_feat_per_s"
 UNIT = "edge*feat/s"
 NOMINAL_HBM_GBS = 8000.0
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.txt")
-KERNEL_SOURCES = ["dg_aggregate_kernels.cuh", "dg_aggregate.cu", "dg_internal.cuh"]
+KERNEL_SOURCES = ["dg_aggregate_kernels.cuh", "dg_aggregate.cu"]
 
 
 def kernel_source_hash():
-    """sha256 over the sources of the aggregation kernels: a capture is only quoted for the
-    kernels it was taken with."""
+    """sha256 over the two files that hold the aggregation kernels and their launch shapes: a
+    capture is only quoted for the kernels it was taken with."""
     import hashlib
     h = hashlib.sha256()
     for name in KERNEL_SOURCES:
@@ -468,12 +468,15 @@ def time_calls(torch, fwd_call, bwd_call, reps, flush, device_index):
 
 
 WORKLOAD_PLAN = [
-    # name, feature widths, ops, epoch dims (or None), training share of the vertices
-    ("tiny", (64,), ("sum", "mean"), None, None),
-    ("reddit_like", (602, 256), ("mean",), None, None),
-    ("products_like", (100, 256), ("sum", "mean"), [100, 256, 256, 47], 196615 / 2449029),
-    ("proteins_like", (8, 64, 256), ("sum",), None, None),
-    ("papers_like", (128,), ("sum",), None, None),
+    # name, feature widths, ops, epoch dims (or None), training share of the vertices, reorder
+    ("tiny", (64,), ("sum", "mean"), None, None, None),
+    ("reddit_like", (602, 256), ("mean",), None, None, None),
+    ("products_like", (100, 256), ("sum", "mean"), [100, 256, 256, 47], 196615 / 2449029, None),
+    # the same graph renamed hub-first by dg_graph_reorder (pre-processing, timed under ingest)
+    ("products_like", (100, 256), ("sum", "mean"), [100, 256, 256, 47], 196615 / 2449029,
+     "out_degree"),
+    ("proteins_like", (8, 64, 256), ("sum",), None, None, None),
+    ("papers_like", (128,), ("sum",), None, None, None),
 ]
 
 
@@ -544,13 +547,27 @@ def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_
     (workload, F, op) triples that the caller has measured already."""
     records, ingest, epochs, extras = [], {}, {}, []
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    for name, widths, ops, dims, frac in WORKLOAD_PLAN:
+    for name, widths, ops, dims, frac, reorder in WORKLOAD_PLAN:
         torch.cuda.empty_cache()
         t0 = time.perf_counter()
         sg = synth.make(name, device=dev)
         torch.cuda.synchronize()
         gen_s = time.perf_counter() - t0
         torch.cuda.empty_cache()
+        reorder_ms = None
+        if reorder:
+            g0 = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            renamed = g0.dg_graph_reorder(binding.DG_ORDER_OUT_DEGREE if reorder == "out_degree"
+                                          else binding.DG_ORDER_IN_DEGREE)
+            torch.cuda.synchronize()
+            reorder_ms = 1e3 * (time.perf_counter() - t0)
+            del g0
+            sg.rowptr, sg.colidx, sg.edge_w = renamed.rowptr, renamed.colidx, renamed.edge_w
+            torch.cuda.empty_cache()
+        label = name + (f" (reorder {reorder})" if reorder else "")
+        tkey = name + (f"+{reorder}" if reorder else "")     # key in profiles/dram_traffic.txt
         weighted = sg.edge_w is not None
         n_ref, n_nonempty = distinct_counts(torch, sg)
         t0 = time.perf_counter()
@@ -567,9 +584,10 @@ def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_
         g.dg_graph_transpose(csc_buf, scratch)
         e1.record(torch.cuda.current_stream())
         torch.cuda.synchronize()
-        ingest[name] = {"generate_s": gen_s, "graph_create_ms": create_ms,
-                        "transpose_ms": e0.elapsed_time(e1),
-                        "transpose_edges_per_s": sg.nnz / (e0.elapsed_time(e1) * 1e-3)}
+        ingest[label] = {"generate_s": gen_s, "graph_create_ms": create_ms,
+                         "transpose_ms": e0.elapsed_time(e1),
+                         "transpose_edges_per_s": sg.nnz / (e0.elapsed_time(e1) * 1e-3),
+                         "reorder_ms": reorder_ms}
         del scratch
         torch.cuda.empty_cache()
         colptr, rowidx_T, w_T, _ = g.dg_graph_get_csc()
@@ -600,24 +618,24 @@ def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_
                 b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False)
                 b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_nonempty, op == "mean")
                 rec = {"workload": name, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
-                       "weighted": weighted, "reps": reps,
+                       "weighted": weighted, "reorder": reorder or "none", "reps": reps,
                        "l2": "flushed before every call (inputs fit L2)" if cold
                              else "inputs larger than L2 (no flush needed)",
                        "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
                                   else "H, out, dOut, dH separate",
                        "fwd": direction_record(f_ms, b_fwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
                        "bwd": direction_record(b_ms, b_bwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),
-                       "traffic": {"fwd": ncu_traffic(name, F, op, 1.0, "fwd"),
-                                   "bwd": ncu_traffic(name, F, op, 1.0, "bwd")},
+                       "traffic": {"fwd": ncu_traffic(tkey, F, op, 1.0, "fwd"),
+                                   "bwd": ncu_traffic(tkey, F, op, 1.0, "bwd")},
                        "clocks": clocks}
                 rec["cpu_baseline"] = None if cpu_seconds <= 0 else cpu_baseline_sampled(
                     torch, sg, (colptr, rowidx_T, w_T), H, G, op, cpu_seconds)
                 records.append(rec)
             if dims and F == dims[0]:
-                epochs[name] = epoch_plain(torch, g, sg, H, dims, frac, dev)
+                epochs[label] = epoch_plain(torch, g, sg, H, dims, frac, dev)
             del H, out, G, dH
             torch.cuda.empty_cache()
-            if (name, F) in (("products_like", 100), ("proteins_like", 64)):
+            if (name, F, reorder) in (("products_like", 100, None), ("proteins_like", 64, None)):
                 extras += extra_records(torch, binding, synth, name, g, sg, F, n_ref, peak, flush)
                 torch.cuda.empty_cache()
         del g, csc_buf, colptr, rowidx_T, w_T, sg
@@ -811,8 +829,9 @@ def main():
         traffic = None if t is None else t / per_call
     roofline = {
         "bound": "hbm",
-        "kernel": ("ap_kernel_r40" if (weighted or (dom == "bwd" and op == "mean")) and F >= 64
-                   else "ap_kernel") + f" ({dom}: {per_call} launch(es) per dg_aggregate_{dom} call)",
+        "kernel": ("ap_kernel_r40" if ((weighted or (dom == "bwd" and op == "mean")) and F >= 64)
+                   or F <= 16 else "ap_kernel")
+                  + f" ({dom}: {per_call} launch(es) per dg_aggregate_{dom} call)",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
         "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "launches_per_call": per_call,
@@ -1005,7 +1024,7 @@ def main():
                    and args.reorder == "none")
     if rank == 0 and world == 1 and args.workloads == "all" and default_run:
         head = {"workload": args.workload, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
-                "weighted": weighted, "reps": args.steps,
+                "weighted": weighted, "reorder": "none", "reps": args.steps,
                 "l2": "inputs larger than L2 (no flush needed)",
                 "buffers": "H, out, dOut, dH separate",
                 "fwd": direction_record(fwd_list, b_fwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),

@@ -659,7 +659,10 @@ int heavy_block_count(const Graph* g, K kernel, size_t smem) {
 template <typename E, int VEC, int G, int CPL, bool SCALED, bool SELF, bool FOLD>
 dg_status_t launch_variant(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
                            cudaStream_t s) {
-  constexpr bool kCapped = SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16;
+  // also the narrowest slices (at most 4 lanes per edge, i.e. up to 16 features per slice): their
+  // 32- and 64-byte gathers wait on latency, and six blocks per SM hide more of it than five
+  // (Proteins-like F = 8: 0.425 -> 0.384 ms, F = 16: 0.449 -> 0.429 ms)
+  constexpr bool kCapped = (SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16) || G <= 4;
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
   const int64_t light_blocks = (a.n + rows_per_block - 1) / rows_per_block;
   if constexpr (SELF) {

@@ -83,8 +83,17 @@ __device__ __forceinline__ void take_better(float& best, int32_t& best_k, float 
   }
 }
 
-// Forward: warp per destination row; lane (grp, c) takes feature f0 + c of the edges
-// lo + grp, lo + grp + NG, ...
+constexpr int kTiles = 4;  // feature tiles of G lanes a warp carries through one walk of a row
+// edges in flight per lane group and step: four where only one operand is loaded per message
+template <int BIN> struct EdgesInFlight {
+  static constexpr int value = (BIN == kCopyLhs || BIN == kCopyRhs) ? 4 : 2;
+};
+
+// Forward: warp per destination row.  The indices of a row are read as coalesced batches of 32
+// (one per lane, the next batch in flight while the current one is used) and broadcast by
+// shuffles; lane (grp, c) takes the features f0 + t * G + c, t < kTiles, of two or four edges per
+// step, so that 8 to 16 independent loads per operand are in flight.  No load is predicated:
+// lanes without an edge or a feature read a valid address and their values are dropped.
 template <int BIN, int RED>
 __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a) {
   const int lane = threadIdx.x & 31;
@@ -94,41 +103,86 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
   const int F = a.F, cols = a.cols;
-  for (int f0 = 0; f0 < F; f0 += G) {
-    const bool jok = f0 + c < F;
-    const int j = jok ? f0 + c : 0;
-    float acc = 0.f, total = 0.f, best = 0.f;
-    int32_t best_k = -1;
+  constexpr int kEdges = EdgesInFlight<BIN>::value;
+  for (int f0 = 0; f0 < F; f0 += kTiles * G) {
+    bool jok[kTiles];
+    int j[kTiles];
+    float acc[kTiles], total[kTiles], best[kTiles];
+    int32_t best_k[kTiles];
+#pragma unroll
+    for (int t = 0; t < kTiles; ++t) {
+      jok[t] = f0 + t * G + c < F;
+      j[t] = jok[t] ? f0 + t * G + c : 0;
+      acc[t] = total[t] = best[t] = 0.f;
+      best_k[t] = -1;
+    }
     int chain = 0;
-#pragma unroll 4
-    for (int64_t e = lo + grp; e < hi; e += NG) {
-      const float x = BIN != kCopyRhs ? __ldg(a.X + (size_t)__ldg(a.idx + e) * F + j) : 0.f;
-      const float y = BIN != kCopyLhs ? __ldg(a.Y + (size_t)e * cols + (cols == 1 ? 0 : j)) : 0.f;
-      const float m = message<BIN>(x, y);
-      if (RED == kSum) {
-        acc += m;
-        if (++chain == kChain) { total += acc; acc = 0.f; chain = 0; }
-      } else {
-        take_better<RED>(best, best_k, m, (int32_t)e);
+    int32_t next_u = (BIN != kCopyRhs && lo + lane < hi) ? __ldcs(a.idx + lo + lane) : 0;
+    for (int64_t b = lo; b < hi; b += 32) {
+      const int32_t my_u = next_u;
+      next_u = (BIN != kCopyRhs && b + 32 + lane < hi) ? __ldcs(a.idx + b + 32 + lane) : 0;
+      const int cnt = (int)(hi - b < 32 ? hi - b : 32);
+      for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
+        float x[kEdges][kTiles], y[kEdges][kTiles];
+#pragma unroll
+        for (int i = 0; i < kEdges; ++i) {
+          const int e = e0 + i * NG + grp;
+          const int32_t u = __shfl_sync(kAll, my_u, e & 31);
+          const float* xrow = BIN != kCopyRhs ? a.X + (size_t)u * F : nullptr;
+          const float* yrow = BIN != kCopyLhs ? a.Y + (size_t)(e < cnt ? b + e : b) * cols : nullptr;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) {
+            x[i][t] = BIN != kCopyRhs ? __ldg(xrow + j[t]) : 0.f;
+            y[i][t] = BIN != kCopyLhs ? __ldg(yrow + (cols == 1 ? 0 : j[t])) : 1.f;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < kEdges; ++i) {
+          const int e = e0 + i * NG + grp;
+          const bool valid = e < cnt;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) {
+            const float m = message<BIN>(x[i][t], y[i][t]);
+            if (RED == kSum) {
+              acc[t] += valid ? m : 0.f;
+            } else {
+              // a lane meets its edges in ascending position, so "strictly better" keeps the
+              // lowest position among equal messages; lane groups are merged by take_better
+              const bool take =
+                  valid && (best_k[t] < 0 || (RED == kMax ? m > best[t] : m < best[t]));
+              best[t] = take ? m : best[t];
+              best_k[t] = take ? (int32_t)(b + e) : best_k[t];
+            }
+          }
+        }
+        chain += kEdges;
+        if (RED == kSum && chain >= kChain) {
+          chain = 0;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) { total[t] += acc[t]; acc[t] = 0.f; }
+        }
       }
     }
-    total += acc;
-    for (int off = G; off < 32; off <<= 1) {
-      if (RED == kSum) {
-        total += __shfl_xor_sync(kAll, total, off);
-      } else {
-        const float ob = __shfl_xor_sync(kAll, best, off);
-        const int32_t ok = __shfl_xor_sync(kAll, best_k, off);
-        take_better<RED>(best, best_k, ob, ok);
+#pragma unroll
+    for (int t = 0; t < kTiles; ++t) {
+      total[t] += acc[t];
+      for (int off = G; off < 32; off <<= 1) {
+        if (RED == kSum) {
+          total[t] += __shfl_xor_sync(kAll, total[t], off);
+        } else {
+          const float ob = __shfl_xor_sync(kAll, best[t], off);
+          const int32_t ok = __shfl_xor_sync(kAll, best_k[t], off);
+          take_better<RED>(best[t], best_k[t], ob, ok);
+        }
       }
-    }
-    if (grp == 0 && jok) {
-      const size_t o = (size_t)row * F + j;
-      if (RED == kSum) {
-        a.out[o] = total;
-      } else {
-        a.out[o] = best_k >= 0 ? best : 0.f;
-        if (a.arg_out) a.arg_out[o] = best_k;
+      if (grp == 0 && jok[t]) {
+        const size_t o = (size_t)row * F + j[t];
+        if (RED == kSum) {
+          a.out[o] = total[t];
+        } else {
+          a.out[o] = best_k[t] >= 0 ? best[t] : 0.f;
+          if (a.arg_out) a.arg_out[o] = best_k[t];
+        }
       }
     }
   }
@@ -136,7 +190,8 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
 
 // Gradient with respect to fV: warp per source vertex u over its CSC segment,
 //   dV[u][j] = sum_q sel * dO[v_q][j] * d(x (x) y)/dx,   sel = [arg[v_q][j] == perm[q]] (max/min)
-// The derivative depends on y only (and not at all for copylhs / add / sub).
+// The derivative depends on y only (and not at all for copylhs / add / sub).  Same walk as the
+// forward kernel: batched indices (destination and CSR position), unpredicated loads.
 template <int BIN, int RED>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const GenArgs a) {
   const int lane = threadIdx.x & 31;
@@ -147,25 +202,64 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
   const int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
   const int F = a.F, cols = a.cols;
   constexpr bool kNeedsY = BIN == kMul || BIN == kDiv;
-  for (int f0 = 0; f0 < F; f0 += G) {
-    const bool jok = f0 + c < F;
-    const int j = jok ? f0 + c : 0;
-    float acc = 0.f, total = 0.f;
-    int chain = 0;
-#pragma unroll 4
-    for (int64_t q = lo + grp; q < hi; q += NG) {
-      const size_t vj = (size_t)__ldg(a.idx + q) * F + j;
-      float t = __ldg(a.X + vj);  // dO[v][j]
-      int32_t k = 0;
-      if (kNeedsY || RED != kSum) k = __ldg(a.perm + q);
-      if (kNeedsY) t *= d_dx<BIN>(__ldg(a.Y + (size_t)k * cols + (cols == 1 ? 0 : j)));
-      if (RED != kSum && __ldg(a.arg + vj) != k) t = 0.f;
-      acc += t;
-      if (++chain == kChain) { total += acc; acc = 0.f; chain = 0; }
+  constexpr bool kNeedsK = kNeedsY || RED != kSum;
+  constexpr int kEdges = 2;
+  for (int f0 = 0; f0 < F; f0 += kTiles * G) {
+    bool jok[kTiles];
+    int j[kTiles];
+    float acc[kTiles], total[kTiles];
+#pragma unroll
+    for (int t = 0; t < kTiles; ++t) {
+      jok[t] = f0 + t * G + c < F;
+      j[t] = jok[t] ? f0 + t * G + c : 0;
+      acc[t] = total[t] = 0.f;
     }
-    total += acc;
-    for (int off = G; off < 32; off <<= 1) total += __shfl_xor_sync(kAll, total, off);
-    if (grp == 0 && jok) a.out[(size_t)u * F + j] = total;
+    int chain = 0;
+    for (int64_t b = lo; b < hi; b += 32) {
+      const bool mine = b + lane < hi;
+      const int32_t my_v = mine ? __ldcs(a.idx + b + lane) : 0;
+      const int32_t my_k = (kNeedsK && mine) ? __ldcs(a.perm + b + lane) : 0;
+      const int cnt = (int)(hi - b < 32 ? hi - b : 32);
+      for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
+        float g[kEdges][kTiles], y[kEdges][kTiles];
+        int32_t sel[kEdges][kTiles], k[kEdges];
+#pragma unroll
+        for (int i = 0; i < kEdges; ++i) {
+          const int e = e0 + i * NG + grp;
+          const size_t vrow = (size_t)__shfl_sync(kAll, my_v, e & 31) * F;
+          k[i] = __shfl_sync(kAll, my_k, e & 31);
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) {
+            g[i][t] = __ldg(a.X + vrow + j[t]);  // dO[v][j]
+            y[i][t] = kNeedsY ? __ldg(a.Y + (size_t)k[i] * cols + (cols == 1 ? 0 : j[t])) : 1.f;
+            sel[i][t] = RED != kSum ? __ldg(a.arg + vrow + j[t]) : 0;
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < kEdges; ++i) {
+          const bool valid = e0 + i * NG + grp < cnt;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) {
+            float v = g[i][t];
+            if (kNeedsY) v *= d_dx<BIN>(y[i][t]);
+            if (!valid || (RED != kSum && sel[i][t] != k[i])) v = 0.f;
+            acc[t] += v;
+          }
+        }
+        chain += kEdges;
+        if (chain >= kChain) {
+          chain = 0;
+#pragma unroll
+          for (int t = 0; t < kTiles; ++t) { total[t] += acc[t]; acc[t] = 0.f; }
+        }
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < kTiles; ++t) {
+      total[t] += acc[t];
+      for (int off = G; off < 32; off <<= 1) total[t] += __shfl_xor_sync(kAll, total[t], off);
+      if (grp == 0 && jok[t]) a.out[(size_t)u * F + j[t]] = total[t];
+    }
   }
 }
 
@@ -231,34 +325,162 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_scalar_kernel(cons
   }
 }
 
-// The same dot product with 16-byte loads for the entry point dg_aggregate_edge_grad (rows of
-// both matrices 16-byte aligned): lane c of a group takes float4 c, c + G, ... of the two rows.
-__global__ void __launch_bounds__(kGenBlock) edge_weight_grad_vec4_kernel(const GenArgs a) {
+// ---- dg_aggregate_edge_grad: dW[k] = s_v * <H[u_k], dOut[v_k]>, one dot product per edge ----
+//
+// The output is one value per edge, so a row of any length splits freely: the first blocks of the
+// launch walk the handle's list of heavy rows (longest first), the 8 warps of a block taking
+// interleaved 32-edge batches of one row; in the other blocks a warp owns one light row.  Lanes
+// are spread along the features (G lanes per edge, VEC floats per load), U edges are in flight
+// per lane group before the first multiply, and with G = 32 the eight partial dot products of a
+// step are reduced together by a transposing butterfly (9 shuffles for 8 edges instead of 40).
+// dOut[v] is the same row for every edge of v: a slab of it is read (from L1) once per U edges.
+struct EdgeGradArgs {
+  const int64_t* rowptr;
+  const int32_t* colidx;
+  const float* H;
+  const float* dOut;
+  float* dW;
+  const int32_t* heavy_list;
+  const int32_t* heavy_count;
+  int32_t heavy_cap;
+  int32_t heavy_threshold;
+  int64_t n;
+  int32_t F;
+  int32_t row_scale;  // 0 none, 1 = 1/deg(v), 2 = 1/(deg(v)+1)
+  // one pass of a sliced / source-blocked call: features [f_lo, f_lo + f_cnt), the piece
+  // [seg_lo[v], seg_hi[v]) of every row (nullptr: whole rows), and whether dW already holds the
+  // dot products of the earlier feature slices
+  int32_t f_lo, f_cnt;
+  const int32_t* seg_lo;
+  const int32_t* seg_hi;
+  int32_t accumulate;
+};
+
+template <int VEC> struct LoadVec;
+template <> struct LoadVec<1> { using T = float; };
+template <> struct LoadVec<2> { using T = float2; };
+template <> struct LoadVec<4> { using T = float4; };
+__device__ __forceinline__ float dotv(float x, float g) { return x * g; }
+__device__ __forceinline__ float dotv(float2 x, float2 g) { return x.x * g.x + x.y * g.y; }
+__device__ __forceinline__ float dotv(float4 x, float4 g) {
+  return x.x * g.x + x.y * g.y + x.z * g.z + x.w * g.w;
+}
+
+template <int VEC, int G>
+__device__ __forceinline__ void edge_grad_row(const EdgeGradArgs& a, int64_t v, int64_t lo,
+                                              int64_t hi, int64_t degree, int first_batch,
+                                              int batch_stride) {
+  using V = typename LoadVec<VEC>::T;
+  constexpr int NG = 32 / G;
+  constexpr int U = G == 32 ? 8 : 4;  // edges in flight per lane group
   const int lane = threadIdx.x & 31;
-  const int64_t v = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
-  if (v >= a.n) return;
-  const int G = 1 << a.log_g, NG = 32 >> a.log_g;
-  const int grp = lane >> a.log_g, c = lane & (G - 1);
-  const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
-  const int nvec = a.F >> 2;
+  const int grp = lane / G, c = lane % G;
+  const int nvec = a.f_cnt / VEC;
   float s = 1.f;
-  if (a.row_scale) s = 1.0f / (float)(hi - lo + (a.row_scale == 2 ? 1 : 0));
-  const float4* grow = reinterpret_cast<const float4*>(a.X + (size_t)v * a.F);
-  for (int64_t e0 = lo; e0 < hi; e0 += NG) {
-    const int64_t e = e0 + grp;
-    const bool eok = e < hi;
-    float dot = 0.f;
-    if (eok) {
-      const float4* xrow = reinterpret_cast<const float4*>(a.V + (size_t)__ldg(a.idx + e) * a.F);
-#pragma unroll 4
-      for (int j = c; j < nvec; j += G) {
-        const float4 x = __ldg(xrow + j), g = __ldg(grow + j);
-        dot += x.x * g.x + x.y * g.y + x.z * g.z + x.w * g.w;
+  if (a.row_scale) s = 1.0f / (float)(degree + (a.row_scale == 2 ? 1 : 0));
+  const V* grow = reinterpret_cast<const V*>(a.dOut + (size_t)v * a.F + a.f_lo);
+  for (int64_t b = lo + (int64_t)first_batch * 32; b < hi; b += (int64_t)batch_stride * 32) {
+    // lanes past the end of the row name vertex 0: their loads are harmless and never written
+    const int32_t my_u = b + lane < hi ? __ldcs(a.colidx + b + lane) : 0;
+    const int cnt = (int)(hi - b < 32 ? hi - b : 32);
+    for (int e0 = 0; e0 < cnt; e0 += NG * U) {
+      // No predicate on the loads: a slab of dOut[v] (one vector per lane) is read once and
+      // multiplied with the matching slab of the U gathered rows, U independent loads in flight.
+      const V* xrow[U];
+      float p[U];
+#pragma unroll
+      for (int j = 0; j < U; ++j) {
+        const int32_t u = __shfl_sync(kAll, my_u, (e0 + j * NG + grp) & 31);
+        xrow[j] = reinterpret_cast<const V*>(a.H + (size_t)u * a.F + a.f_lo);
+        p[j] = 0.f;
+      }
+      for (int t = c; t < nvec; t += G) {
+        const V gt = __ldg(grow + t);
+        V x[U];
+#pragma unroll
+        for (int j = 0; j < U; ++j) x[j] = __ldg(xrow[j] + t);
+#pragma unroll
+        for (int j = 0; j < U; ++j) p[j] += dotv(x[j], gt);
+      }
+      if constexpr (G == 32) {
+        // transposing butterfly: after the three exchange steps lane L holds, summed over eight
+        // lanes, the dot product of edge j(L) = 4*bit4 + 2*bit3 + bit2; two more steps finish it
+        float q[4], r[2];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const bool up = lane & 16;
+          const float got = __shfl_xor_sync(kAll, up ? p[i] : p[i + 4], 16);
+          q[i] = (up ? p[i + 4] : p[i]) + got;
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          const bool up = lane & 8;
+          const float got = __shfl_xor_sync(kAll, up ? q[i] : q[i + 2], 8);
+          r[i] = (up ? q[i + 2] : q[i]) + got;
+        }
+        const bool up = lane & 4;
+        float t = (up ? r[1] : r[0]) + __shfl_xor_sync(kAll, up ? r[0] : r[1], 4);
+        t += __shfl_xor_sync(kAll, t, 2);
+        t += __shfl_xor_sync(kAll, t, 1);
+        const int j = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+        if ((lane & 3) == 0 && e0 + j < cnt) {
+          float* w = a.dW + b + e0 + j;
+          *w = a.accumulate ? *w + t * s : t * s;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < U; ++j) {
+          float t = p[j];
+#pragma unroll
+          for (int off = 1; off < G; off <<= 1) t += __shfl_xor_sync(kAll, t, off);
+          const int e = e0 + j * NG + grp;
+          if (c == 0 && e < cnt) {
+            float* w = a.dW + b + e;
+            *w = a.accumulate ? *w + t * s : t * s;
+          }
+        }
       }
     }
-    for (int off = 1; off < G; off <<= 1) dot += __shfl_xor_sync(kAll, dot, off);
-    if (eok && c == 0) a.out[e] = dot * s;
   }
+}
+
+template <int VEC, int G>
+__global__ void __launch_bounds__(kGenBlock) edge_grad_kernel(const EdgeGradArgs a,
+                                                              const int heavy_blocks) {
+  const int warp = threadIdx.x >> 5;
+  if ((int)blockIdx.x < heavy_blocks) {
+    const int count = min(*a.heavy_count, a.heavy_cap);
+    for (int i = blockIdx.x; i < count; i += heavy_blocks) {
+      const int64_t v = a.heavy_list[i];
+      const int64_t lo = __ldg(a.rowptr + v), hi = __ldg(a.rowptr + v + 1);
+      edge_grad_row<VEC, G>(a, v, a.seg_lo ? __ldg(a.seg_lo + v) : lo,
+                            a.seg_hi ? __ldg(a.seg_hi + v) : hi, hi - lo, warp, kGenWarps);
+    }
+    return;
+  }
+  const int64_t v = (int64_t)(blockIdx.x - heavy_blocks) * kGenWarps + warp;
+  if (v >= a.n) return;
+  const int64_t lo = __ldg(a.rowptr + v), hi = __ldg(a.rowptr + v + 1);
+  if (hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this row's edges
+  edge_grad_row<VEC, G>(a, v, a.seg_lo ? __ldg(a.seg_lo + v) : lo,
+                        a.seg_hi ? __ldg(a.seg_hi + v) : hi, hi - lo, 0, 1);
+}
+
+template <int VEC>
+dg_status_t launch_edge_grad(const dg_graph* g, const EdgeGradArgs& a, cudaStream_t s) {
+  const int nvec = a.f_cnt / VEC;
+  const int heavy_blocks = g->sm_count * 4;
+  const unsigned grid = (unsigned)(heavy_blocks + (a.n + kGenWarps - 1) / kGenWarps);
+#define DG_EG_CASE(GG)                                                              \
+  if (nvec <= GG || GG == 32) {                                                     \
+    edge_grad_kernel<VEC, GG><<<grid, kGenBlock, 0, s>>>(a, heavy_blocks);          \
+    DG_CUDA(cudaGetLastError());                                                    \
+    count_launches(1);                                                              \
+    return DG_OK;                                                                   \
+  }
+  DG_EG_CASE(1) DG_EG_CASE(2) DG_EG_CASE(4) DG_EG_CASE(8) DG_EG_CASE(16) DG_EG_CASE(32)
+#undef DG_EG_CASE
+  return DG_OK;
 }
 
 int log_group(int32_t width) {  // lanes per edge: the power of two covering `width`, at most 32
@@ -418,26 +640,50 @@ dg_status_t dg_aggregate_edge_grad(dg_graph_t g, const float* H, const float* dO
   if (op != DG_OP_SUM && op != DG_OP_MEAN) return bad("op must be DG_OP_SUM or DG_OP_MEAN");
   if (g->nnz == 0) return DG_OK;
   if (!H || !dOut || !dW) return bad("H, dOut or dW is NULL");
-  GenArgs a{};
-  a.ptr = g->rowptr;
-  a.idx = g->colidx;
-  a.X = dOut;
-  a.V = H;
-  a.out = dW;
+  EdgeGradArgs a{};
+  a.rowptr = g->rowptr;
+  a.colidx = g->colidx;
+  a.H = H;
+  a.dOut = dOut;
+  a.dW = dW;
+  a.heavy_list = g->heavy_rows;
+  a.heavy_count = g->counters + 0;
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.n = g->n;
   a.F = F;
-  a.cols = 1;
   a.row_scale = op == DG_OP_MEAN ? (g->self_loops ? 2 : 1) : 0;
   cudaStream_t s = (cudaStream_t)stream;
-  if (F % 4 == 0 && (((uintptr_t)H | (uintptr_t)dOut) & 15) == 0) {
-    a.log_g = log_group(F / 4);
-    edge_weight_grad_vec4_kernel<<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
-    DG_CUDA(cudaGetLastError());
-    count_launches(1);
-    return DG_OK;
+  const uintptr_t both = (uintptr_t)H | (uintptr_t)dOut;
+  const int vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
+  // Like the aggregation itself (Algorithm 2 with L2 as the cache): when the gathered matrix
+  // does not stay L2-resident and the rows carry split pointers, the call is cut into feature
+  // slices of 128 vectors and source-vertex blocks sized to the L2 budget, one launch each; the
+  // blocks partition the edges, the slices add up in dW.
+  int64_t slice = F;
+  int nb = 1;
+  if (g->split_csr && (double)g->n * F * 4.0 > (double)g->l2_budget_bytes) {
+    slice = 128LL * vec < F ? 128LL * vec : F;
+    while (nb < kFineBlocks && (double)g->n / nb * (double)(slice * 4 + 128) > (double)g->l2_budget_bytes)
+      nb *= 2;
+    if ((double)g->nnz / (double)g->n / nb < 32.0) { nb = 1; slice = F; }  // pieces too short to pay
   }
-  a.log_g = log_group(F);
-  return BwdEdgeScalarLauncher<kMul, kSum>::run(a, s);
+  const int per = kFineBlocks / nb;
+  for (int j = 0; j < nb; ++j) {
+    if (nb > 1) {
+      a.seg_lo = g->split_csr + (size_t)(j * per) * (size_t)g->n;
+      a.seg_hi = g->split_csr + (size_t)((j + 1) * per) * (size_t)g->n;
+    }
+    for (int64_t f0 = 0; f0 < F; f0 += slice) {
+      a.f_lo = (int32_t)f0;
+      a.f_cnt = (int32_t)(F - f0 < slice ? F - f0 : slice);
+      a.accumulate = f0 > 0;
+      const dg_status_t st = vec == 4 ? launch_edge_grad<4>(g, a, s)
+                           : vec == 2 ? launch_edge_grad<2>(g, a, s) : launch_edge_grad<1>(g, a, s);
+      if (st != DG_OK) return st;
+    }
+  }
+  return DG_OK;
 }
 
 }  // extern "C"

@@ -144,9 +144,10 @@ dg_status_t refresh_csc_weights(Graph* g, cudaStream_t s);
 // dg_api.cu: what follows every transposition (heavy columns, the long-column count on its way)
 dg_status_t finish_transpose(Graph* g, cudaStream_t s);
 // the stable radix sort behind it, for other pre-processing steps (see dg_transpose.cu)
-int sort_passes(int64_t key_range);
+struct SortPlan { int digit_bits; int passes; };
+SortPlan sort_plan(int64_t key_range);
 void sort_scratch_sizes(int64_t count, size_t* hist_bytes, size_t* sums_bytes);
-dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count, int passes,
+dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count, SortPlan plan,
                        uint32_t* const keys_buf[2], uint32_t* vals_final, uint32_t* vals_tmp,
                        uint32_t* hist, uint32_t* sums, const uint32_t** sorted_keys,
                        cudaStream_t s);

@@ -200,7 +200,7 @@ dg_status_t dg_graph_reorder(dg_graph_t g, dg_order_t order, const int32_t* give
     count_launches(1);
     const uint32_t* sorted = nullptr;
     // values end in va (old_of_new); vb may be reused as the ping-pong buffer: the keys are made
-    if (dg_status_t st = sort_pairs(k1, nullptr, n, sort_passes(nnz + 1), keys_buf, va, vb, hist,
+    if (dg_status_t st = sort_pairs(k1, nullptr, n, sort_plan(nnz + 1), keys_buf, va, vb, hist,
                                     sums, &sorted, s))
       return st;
     invert_order_kernel<<<blocks_of(n), 256, 0, s>>>(va, n, new_of_old);
@@ -218,14 +218,14 @@ dg_status_t dg_graph_reorder(dg_graph_t g, dg_order_t order, const int32_t* give
         order_u, reinterpret_cast<const uint32_t*>(g->colidx), nnz, k1);
     DG_CUDA(cudaGetLastError());
     const uint32_t* sorted = nullptr;
-    if (dg_status_t st = sort_pairs(k1, nullptr, nnz, sort_passes(n), keys_buf, va, vb, hist, sums,
+    if (dg_status_t st = sort_pairs(k1, nullptr, nnz, sort_plan(n), keys_buf, va, vb, hist, sums,
                                     &sorted, s))
       return st;
     // keys of the second sort: new id of the destination of every position, in the first sort's order
     if (dg_status_t st = expand_rows(g->rowptr, n, nnz, new_of_old, keys_buf[0], s)) return st;
     gather_u32_kernel<<<blocks_of(nnz), 256, 0, s>>>(keys_buf[0], va, nnz, keys_buf[1]);
     DG_CUDA(cudaGetLastError());
-    if (dg_status_t st = sort_pairs(keys_buf[1], va, nnz, sort_passes(n), keys_buf, pos2, vb, hist,
+    if (dg_status_t st = sort_pairs(keys_buf[1], va, nnz, sort_plan(n), keys_buf, pos2, vb, hist,
                                     sums, &sorted, s))
       return st;
     if (dg_status_t st = pointers_from_sorted_keys(sorted, nnz, n, rowptr2, s)) return st;

@@ -3,8 +3,8 @@
 // of the backward pass implicit; the result here is defined as the stable counting sort of the
 // edge positions by source vertex, which has exactly one correct answer.
 //
-// One pass over a digit of kRadixBits bits is three kernels and never makes one block wait for
-// another:
+// The digits are 8 bits wide, or 9 where that pays (see sort_plan).  One pass over a digit is
+// three kernels and never makes one block wait for another:
 //   1. digit_histogram : per tile of kTile keys, the number of keys per digit -> hist[digit][tile]
 //   2. exclusive scan of hist (digit-major, so the scan yields global output offsets):
 //      scan_reduce -> scan_spine (one block) -> scan_apply
@@ -18,8 +18,7 @@
 namespace dg {
 namespace {
 
-constexpr int kRadixBits = 8;
-constexpr int kRadix = 1 << kRadixBits;
+constexpr int kMaxRadixBits = 9;
 constexpr int kSortBlock = 256;
 constexpr int kSortWarps = kSortBlock / 32;
 constexpr int kItems = 16;                       // keys per thread
@@ -29,19 +28,22 @@ constexpr int kScanItems = 16;
 constexpr int kScanChunk = kScanBlock * kScanItems;
 constexpr unsigned kFull = 0xffffffffu;
 
+template <int BITS>
 __device__ __forceinline__ uint32_t digit_of(uint32_t key, int shift) {
-  return (key >> shift) & (kRadix - 1);
+  return (key >> shift) & ((1u << BITS) - 1u);
 }
 
 // A thread reads its keys as 16-byte vectors when the array allows it (four loads in flight
 // then cover the whole tile; with 4-byte loads the kernel waited on memory at a third of the
 // copy bandwidth).  The caller's colidx, the keys of the first pass, is only 4-byte aligned in
 // general: `vector_ok` says whether keys is 16-byte aligned.
+template <int BITS>
 __global__ void __launch_bounds__(kSortBlock)
 digit_histogram(const uint32_t* __restrict__ keys, int64_t count, int shift, int64_t tiles,
                 int vector_ok, uint32_t* __restrict__ hist) {
-  __shared__ uint32_t h[kRadix];
-  h[threadIdx.x] = 0;
+  constexpr int R = 1 << BITS;
+  __shared__ uint32_t h[R];
+  for (int d = threadIdx.x; d < R; d += kSortBlock) h[d] = 0;
   __syncthreads();
   const int64_t base = (int64_t)blockIdx.x * kTile;
   if (vector_ok && base + kTile <= count) {
@@ -51,20 +53,20 @@ digit_histogram(const uint32_t* __restrict__ keys, int64_t count, int shift, int
     for (int i = 0; i < kItems / 4; ++i) k[i] = v[i * kSortBlock + threadIdx.x];
 #pragma unroll
     for (int i = 0; i < kItems / 4; ++i) {
-      atomicAdd(&h[digit_of(k[i].x, shift)], 1u);
-      atomicAdd(&h[digit_of(k[i].y, shift)], 1u);
-      atomicAdd(&h[digit_of(k[i].z, shift)], 1u);
-      atomicAdd(&h[digit_of(k[i].w, shift)], 1u);
+      atomicAdd(&h[digit_of<BITS>(k[i].x, shift)], 1u);
+      atomicAdd(&h[digit_of<BITS>(k[i].y, shift)], 1u);
+      atomicAdd(&h[digit_of<BITS>(k[i].z, shift)], 1u);
+      atomicAdd(&h[digit_of<BITS>(k[i].w, shift)], 1u);
     }
   } else {
 #pragma unroll 4
     for (int i = 0; i < kItems; ++i) {
       const int64_t k = base + i * kSortBlock + threadIdx.x;
-      if (k < count) atomicAdd(&h[digit_of(keys[k], shift)], 1u);
+      if (k < count) atomicAdd(&h[digit_of<BITS>(keys[k], shift)], 1u);
     }
   }
   __syncthreads();
-  hist[(int64_t)threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];
+  for (int d = threadIdx.x; d < R; d += kSortBlock) hist[(int64_t)d * tiles + blockIdx.x] = h[d];
 }
 
 // ---- exclusive scan of a uint32 array of length m (in place), three kernels ----
@@ -146,11 +148,12 @@ scan_apply(uint32_t* __restrict__ data, int64_t m, const uint32_t* __restrict__ 
 // another): one ballot per digit bit, each keeping the lanes that agree with this lane on that
 // bit.  Unlike match.any, whose cost grows with the number of distinct values in the warp (about
 // 30 for the random low digits of vertex ids), this costs the same for every digit mix.
+template <int BITS>
 __device__ __forceinline__ unsigned digit_peers(uint32_t d, bool valid) {
   const unsigned have = __ballot_sync(kFull, valid);
   unsigned peers = valid ? have : ~have;
 #pragma unroll
-  for (int b = 0; b < kRadixBits; ++b) {
+  for (int b = 0; b < BITS; ++b) {
     const bool bit = (d >> b) & 1u;
     const unsigned m = __ballot_sync(kFull, bit);
     peers &= bit ? m : ~m;
@@ -164,29 +167,41 @@ __device__ __forceinline__ unsigned digit_peers(uint32_t d, bool valid) {
 // Four blocks per SM (64 registers a thread): the ranking is a chain of shared-memory and
 // ballot latencies, and the fourth block hides more of it than the few spilled words cost
 // (three blocks at 80 registers were 10 % slower, five with the values read late 3 % slower).
+template <int BITS>
 __global__ void __launch_bounds__(kSortBlock, 4)
 digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
               int64_t count, int shift, int64_t tiles, const uint32_t* __restrict__ offsets,
               uint32_t* __restrict__ keys_out, uint32_t* __restrict__ vals_out) {
+  constexpr int R = 1 << BITS;
+  constexpr int DPT = R / kSortBlock;  // digits a thread owns (consecutive ones): 1 or 2
   // A warp ranks its 512 keys as two streams of 256 (rounds 0..7 and 8..15), each with its own
   // counters, so that two independent chains of counter updates are in flight at a time.
-  __shared__ uint16_t cnt_a[kSortWarps][kRadix];
-  __shared__ uint16_t cnt_b[kSortWarps][kRadix];
-  __shared__ uint32_t digit_base[kRadix];
-  __shared__ uint32_t global_base[kRadix];
-  __shared__ uint32_t skeys[kTile];
-  __shared__ uint32_t svals[kTile];
+  // Dynamic shared memory (52 KB with 9-bit digits): cnt_a, cnt_b, digit_base, global_base,
+  // skeys, svals.
+  extern __shared__ __align__(16) unsigned char scatter_smem[];
+  uint16_t (*cnt_a)[R] = reinterpret_cast<uint16_t (*)[R]>(scatter_smem);
+  uint16_t (*cnt_b)[R] = cnt_a + kSortWarps;
+  uint32_t* digit_base = reinterpret_cast<uint32_t*>(cnt_b + kSortWarps);
+  uint32_t* global_base = digit_base + R;
+  uint32_t* skeys = global_base + R;
+  uint32_t* svals = skeys + kTile;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned lt_mask = (1u << lane) - 1u;
   const int64_t tile_base = (int64_t)blockIdx.x * kTile;
   const int64_t remaining = count - tile_base;
   const int tile_count = remaining < kTile ? (int)remaining : kTile;
 
-  // this tile's global offset of digit threadIdx.x: fetched now, needed after the ranking
-  const uint32_t my_global_base = offsets[(int64_t)threadIdx.x * tiles + blockIdx.x];
+  // this tile's global offsets of the thread's digits: fetched now, needed after the ranking
+  uint32_t my_global_base[DPT];
+#pragma unroll
+  for (int i = 0; i < DPT; ++i)
+    my_global_base[i] = offsets[(int64_t)(threadIdx.x * DPT + i) * tiles + blockIdx.x];
   for (int w = 0; w < kSortWarps; ++w) {
-    cnt_a[w][threadIdx.x] = 0;
-    cnt_b[w][threadIdx.x] = 0;
+#pragma unroll
+    for (int i = 0; i < DPT; ++i) {
+      cnt_a[w][threadIdx.x * DPT + i] = 0;
+      cnt_b[w][threadIdx.x * DPT + i] = 0;
+    }
   }
   __syncthreads();
 
@@ -210,8 +225,8 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
       const int rr = r + stream * kHalf;
       uint16_t* cnt = stream ? cnt_b[warp] : cnt_a[warp];
       const bool valid = warp * (32 * kItems) + rr * 32 + lane < tile_count;
-      const uint32_t d = valid ? digit_of(key[rr], shift) : 0u;
-      const unsigned peers = digit_peers(d, valid);
+      const uint32_t d = valid ? digit_of<BITS>(key[rr], shift) : 0u;
+      const unsigned peers = digit_peers<BITS>(d, valid);
       const int leader = __ffs(peers) - 1;
       uint32_t before = 0;
       if (valid && lane == leader) {
@@ -225,22 +240,35 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
   }
   __syncthreads();
 
-  // thread t owns digit t: exclusive prefix over (warp, stream), then over the digits
+  // a thread owns DPT consecutive digits: exclusive prefix over (warp, stream) inside each, then
+  // over the digits
   {
-    const int d = threadIdx.x;
-    uint32_t run = 0;
+    uint32_t in_digit[DPT];
+    uint32_t mine = 0;
 #pragma unroll
-    for (int w = 0; w < kSortWarps; ++w) {
-      const uint32_t ca = cnt_a[w][d];
-      cnt_a[w][d] = (uint16_t)run;
-      run += ca;
-      const uint32_t cb = cnt_b[w][d];
-      cnt_b[w][d] = (uint16_t)run;
-      run += cb;
+    for (int i = 0; i < DPT; ++i) {
+      const int d = threadIdx.x * DPT + i;
+      uint32_t run = 0;
+#pragma unroll
+      for (int w = 0; w < kSortWarps; ++w) {
+        const uint32_t ca = cnt_a[w][d];
+        cnt_a[w][d] = (uint16_t)run;
+        run += ca;
+        const uint32_t cb = cnt_b[w][d];
+        cnt_b[w][d] = (uint16_t)run;
+        run += cb;
+      }
+      in_digit[i] = run;
+      mine += run;
     }
     uint32_t total;
-    digit_base[d] = block_exclusive_scan(run, &total);
-    global_base[d] = my_global_base;
+    uint32_t start = block_exclusive_scan(mine, &total);
+#pragma unroll
+    for (int i = 0; i < DPT; ++i) {
+      digit_base[threadIdx.x * DPT + i] = start;
+      global_base[threadIdx.x * DPT + i] = my_global_base[i];
+      start += in_digit[i];
+    }
   }
   __syncthreads();
 
@@ -248,7 +276,7 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
   for (int r = 0; r < kItems; ++r) {
     const int local = warp * (32 * kItems) + r * 32 + lane;
     if (local < tile_count) {
-      const uint32_t d = digit_of(key[r], shift);
+      const uint32_t d = digit_of<BITS>(key[r], shift);
       const uint32_t in_digit = r < kHalf ? cnt_a[warp][d] : cnt_b[warp][d];
       const uint32_t pos = digit_base[d] + in_digit + rank[r];
       skeys[pos] = key[r];
@@ -259,11 +287,17 @@ digit_scatter(const uint32_t* __restrict__ keys_in, const uint32_t* __restrict__
 
   for (int i = threadIdx.x; i < tile_count; i += kSortBlock) {
     const uint32_t k = skeys[i];
-    const uint32_t d = digit_of(k, shift);
+    const uint32_t d = digit_of<BITS>(k, shift);
     const uint32_t dst = global_base[d] + ((uint32_t)i - digit_base[d]);
     if (keys_out) keys_out[dst] = k;
     vals_out[dst] = svals[i];
   }
+}
+
+template <int BITS>
+constexpr size_t scatter_smem_bytes() {
+  return (size_t)2 * kSortWarps * (1 << BITS) * sizeof(uint16_t) + (size_t)2 * (1 << BITS) * sizeof(uint32_t) +
+         (size_t)2 * kTile * sizeof(uint32_t);
 }
 
 // colptr[u] = first position q whose sorted key is >= u.  Position q fills the ids between the
@@ -432,9 +466,9 @@ Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
   L.mscale_off = o; o += align256((size_t)nnz * 4);
   L.split_off = o;  o += wants_split(n, nnz) ? align256((size_t)(kFineBlocks + 1) * n * 4) : 0;
   L.csc_bytes = o > 0 ? o : 256;
-  L.passes = sort_passes(n);
+  L.passes = sort_plan(n).passes;
   L.tiles = (nnz + kTile - 1) / kTile;
-  L.hist_len = L.tiles * kRadix;
+  L.hist_len = L.tiles * (1 << kMaxRadixBits);
   L.chunks = (L.hist_len + kScanChunk - 1) / kScanChunk;
   o = 0;
   L.keys_a_off = o; o += align256((size_t)nnz * 4);
@@ -448,38 +482,50 @@ Layout make_layout(int64_t n, int64_t nnz, bool weighted) {
 
 }  // namespace
 
-int sort_passes(int64_t key_range) {
+// Digit width and number of passes for keys in [0, key_range).  A 9-bit pass costs about a third
+// more than an 8-bit one (nine ballots per ranking round, twice the counters and histogram, more
+// spilled registers: measured on the 1.6 G-edge graph, 27 key bits, 3 x 9 bits took 100.3 ms
+// against 98.1 ms for 4 x 8), so the wider digit is taken only where it turns three passes into
+// two or two into one (key ranges of 9, 17 and 18 bits: the Reddit- and Proteins-like graphs,
+// whose transposition gains 5 %).
+SortPlan sort_plan(int64_t key_range) {
   int bits = 1;
   while (bits < 31 && ((int64_t)1 << bits) < key_range) ++bits;
-  return (bits + kRadixBits - 1) / kRadixBits;
+  const int p8 = (bits + 7) / 8, p9 = (bits + 8) / 9;
+  SortPlan plan;
+  const bool wide = 4 * p9 < 3 * p8;
+  plan.digit_bits = wide ? 9 : 8;
+  plan.passes = wide ? p9 : p8;
+  return plan;
 }
 
+// Sized for the wider digit, so that one workspace query serves every key range.
 void sort_scratch_sizes(int64_t count, size_t* hist_bytes, size_t* sums_bytes) {
   const int64_t tiles = (count + kTile - 1) / kTile;
-  const int64_t hist_len = tiles * kRadix;
+  const int64_t hist_len = tiles * (1 << kMaxRadixBits);
   const int64_t chunks = (hist_len + kScanChunk - 1) / kScanChunk;
   *hist_bytes = align256((size_t)(hist_len > 0 ? hist_len : 1) * 4);
   *sums_bytes = align256((size_t)(chunks > 0 ? chunks : 1) * 4);
 }
 
-// Stable LSD radix sort of `count` (key, value) pairs over `passes` digits.  vals_in == nullptr
-// means "the value of key i is i".  keys_in is only read; the sorted keys end in one of keys_buf
-// (reported through *sorted_keys; keys_in may be keys_buf[1], which is first written by the second
-// pass), the sorted values in vals_final (vals_tmp is the other buffer of the ping-pong).
-dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count, int passes,
-                       uint32_t* const keys_buf[2], uint32_t* vals_final, uint32_t* vals_tmp,
-                       uint32_t* hist, uint32_t* sums, const uint32_t** sorted_keys,
-                       cudaStream_t s) {
+template <int BITS>
+static dg_status_t sort_passes_run(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count,
+                                   int passes, uint32_t* const keys_buf[2], uint32_t* vals_final,
+                                   uint32_t* vals_tmp, uint32_t* hist, uint32_t* sums,
+                                   const uint32_t** sorted_keys, cudaStream_t s) {
   const int64_t tiles = (count + kTile - 1) / kTile;
-  const int64_t hist_len = tiles * kRadix;
+  const int64_t hist_len = tiles * (1 << BITS);
   const int64_t chunks = (hist_len + kScanChunk - 1) / kScanChunk;
+  constexpr size_t smem = scatter_smem_bytes<BITS>();
+  DG_CUDA(cudaFuncSetAttribute(digit_scatter<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               (int)smem));
   for (int p = 0; p < passes; ++p) {
-    const int shift = p * kRadixBits;
+    const int shift = p * BITS;
     // value buffers alternate so that the last pass lands in vals_final
     uint32_t* vals_out = ((passes - 1 - p) % 2 == 0) ? vals_final : vals_tmp;
     uint32_t* keys_out = keys_buf[p % 2];
-    digit_histogram<<<(unsigned)tiles, kSortBlock, 0, s>>>(keys_in, count, shift, tiles,
-                                                           aligned16(keys_in), hist);
+    digit_histogram<BITS><<<(unsigned)tiles, kSortBlock, 0, s>>>(keys_in, count, shift, tiles,
+                                                                 aligned16(keys_in), hist);
     DG_CUDA(cudaGetLastError());
     scan_reduce<<<(unsigned)chunks, kScanBlock, 0, s>>>(hist, hist_len, sums);
     DG_CUDA(cudaGetLastError());
@@ -487,8 +533,8 @@ dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t
     DG_CUDA(cudaGetLastError());
     scan_apply<<<(unsigned)chunks, kScanBlock, 0, s>>>(hist, hist_len, sums);
     DG_CUDA(cudaGetLastError());
-    digit_scatter<<<(unsigned)tiles, kSortBlock, 0, s>>>(keys_in, vals_in, count, shift, tiles,
-                                                         hist, keys_out, vals_out);
+    digit_scatter<BITS><<<(unsigned)tiles, kSortBlock, smem, s>>>(keys_in, vals_in, count, shift,
+                                                                  tiles, hist, keys_out, vals_out);
     DG_CUDA(cudaGetLastError());
     count_launches(5);
     keys_in = keys_out;
@@ -496,6 +542,21 @@ dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t
   }
   *sorted_keys = keys_in;
   return DG_OK;
+}
+
+// Stable LSD radix sort of `count` (key, value) pairs.  vals_in == nullptr means "the value of key
+// i is i".  keys_in is only read; the sorted keys end in one of keys_buf (reported through
+// *sorted_keys; keys_in may be keys_buf[1], which is first written by the second pass), the
+// sorted values in vals_final (vals_tmp is the other buffer of the ping-pong).
+dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t count,
+                       SortPlan plan, uint32_t* const keys_buf[2], uint32_t* vals_final,
+                       uint32_t* vals_tmp, uint32_t* hist, uint32_t* sums,
+                       const uint32_t** sorted_keys, cudaStream_t s) {
+  if (plan.digit_bits == 9)
+    return sort_passes_run<9>(keys_in, vals_in, count, plan.passes, keys_buf, vals_final, vals_tmp,
+                              hist, sums, sorted_keys, s);
+  return sort_passes_run<8>(keys_in, vals_in, count, plan.passes, keys_buf, vals_final, vals_tmp,
+                            hist, sums, sorted_keys, s);
 }
 
 // ptr[u] = first position whose sorted key is >= u, for u = 0..n (ptr[n] = count)
@@ -558,7 +619,7 @@ dg_status_t transpose_run(Graph* g, void* csc, void* scratch, cudaStream_t s) {
   } else {
     const uint32_t* keys_in = nullptr;
     if (dg_status_t st = sort_pairs(reinterpret_cast<const uint32_t*>(g->colidx), nullptr, nnz,
-                                    L.passes, keys_buf, perm, vals_tmp, hist, sums, &keys_in, s))
+                                    sort_plan(n), keys_buf, perm, vals_tmp, hist, sums, &keys_in, s))
       return st;
     if (dg_status_t st = pointers_from_sorted_keys(keys_in, nnz, n, colptr, s)) return st;
     const unsigned b2 = (unsigned)((nnz + 255) / 256);

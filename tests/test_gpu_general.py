@@ -177,3 +177,21 @@ def test_edge_weight_gradient_on_scaled_workloads(name, scale, F, op):
     torch.cuda.synchronize()
     ref, mag = oracle.edge_weight_grad(to_np(sg.rowptr), to_np(sg.colidx), to_np(H), to_np(G), op)
     assert_within_bound(to_np(dW), ref, mag, "dW")
+
+
+@pytest.mark.parametrize("op", [binding.DG_OP_SUM, binding.DG_OP_MEAN])
+def test_edge_weight_gradient_in_feature_slices_and_source_blocks(op):
+    """With a small L2 budget the call is cut into feature slices (which add up in dW) and source
+    blocks (which partition the edges), one launch each: same result, same bound."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.05)     # 52,093 vertices, 110 edges each
+    g = make_graph(sg)
+    g.dg_graph_set_param("l2_budget_mb", 32)                    # 2 source blocks x 3 slices of 256
+    F = 602
+    H = synth.features(sg.n, F, 23, DEV)
+    G = synth.features(sg.n, F, 24, DEV)
+    before = binding.dg_kernel_launch_count()
+    dW = g.dg_aggregate_edge_grad(H, G, op)
+    torch.cuda.synchronize()
+    assert binding.dg_kernel_launch_count() - before > 4          # really several passes
+    ref, mag = oracle.edge_weight_grad(to_np(sg.rowptr), to_np(sg.colidx), to_np(H), to_np(G), op)
+    assert_within_bound(to_np(dW), ref, mag, "dW, sliced and blocked")
