@@ -44,6 +44,7 @@ struct GenArgs {
   int32_t F, cols;
   int32_t log_g;         // lanes per edge = 1 << log_g
   int32_t row_scale;     // edge-weight gradient: 0 none, 1 = 1/deg(v), 2 = 1/(deg(v)+1)
+  int32_t vec;           // forward: floats per load, 4 or 2 when F and the operands' alignment allow
 };
 
 // one fp32 IEEE operation, never contracted into a neighbouring add
@@ -91,11 +92,18 @@ template <int BIN> struct EdgesInFlight {
 
 // Forward: warp per destination row.  The indices of a row are read as coalesced batches of 32
 // (one per lane, the next batch in flight while the current one is used) and broadcast by
-// shuffles; lane (grp, c) takes the features f0 + t * G + c, t < kTiles, of two or four edges per
-// step, so that 8 to 16 independent loads per operand are in flight.  No load is predicated:
-// lanes without an edge or a feature read a valid address and their values are dropped.
-template <int BIN, int RED>
+// shuffles.  A lane holds four values of a message per edge: with VEC = 4 one 16-byte vector of
+// consecutive features (F a multiple of 4, 16-byte aligned matrices), with VEC = 2 two 8-byte
+// vectors G apart, with VEC = 1 four features G apart; G lanes cover 4 G features per pass, and
+// vectors that lie beyond F are skipped for the whole warp.  Two or four edges per lane group are in flight per step.  No load is
+// predicated per lane: lanes without an edge or a feature read a valid address and their values
+// are dropped.
+template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a) {
+  constexpr int kT = kTiles / VEC;  // vectors per lane and edge (4, 2 or 1)
+  constexpr int NV = kT * VEC;      // values per lane and edge: always 4
+  // edges in flight per lane group and step: four where a message needs one vector load only
+  constexpr int kEdges = (VEC > 1 && EdgesInFlight<BIN>::value == 4) ? 4 : 2;
   const int lane = threadIdx.x & 31;
   const int64_t row = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
   if (row >= a.n) return;
@@ -103,18 +111,21 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
   const int F = a.F, cols = a.cols;
-  constexpr int kEdges = EdgesInFlight<BIN>::value;
-  for (int f0 = 0; f0 < F; f0 += kTiles * G) {
-    bool jok[kTiles];
-    int j[kTiles];
-    float acc[kTiles], total[kTiles], best[kTiles];
-    int32_t best_k[kTiles];
+  for (int f0 = 0; f0 < F; f0 += kT * G * VEC) {
+    bool ok[kT], tile_on[kT];
+    int base[kT];  // first feature of the lane's vector t (0 when it lies beyond F)
+    float acc[NV], total[NV], best[NV];
+    int32_t best_k[NV];
 #pragma unroll
-    for (int t = 0; t < kTiles; ++t) {
-      jok[t] = f0 + t * G + c < F;
-      j[t] = jok[t] ? f0 + t * G + c : 0;
-      acc[t] = total[t] = best[t] = 0.f;
-      best_k[t] = -1;
+    for (int t = 0; t < kT; ++t) {
+      tile_on[t] = f0 + t * G * VEC < F;             // the same for the whole warp
+      ok[t] = f0 + (t * G + c) * VEC < F;
+      base[t] = ok[t] ? f0 + (t * G + c) * VEC : 0;
+    }
+#pragma unroll
+    for (int q = 0; q < NV; ++q) {
+      acc[q] = total[q] = best[q] = 0.f;
+      best_k[q] = -1;
     }
     int chain = 0;
     int32_t next_u = (BIN != kCopyRhs && lo + lane < hi) ? __ldcs(a.idx + lo + lane) : 0;
@@ -123,17 +134,38 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
       next_u = (BIN != kCopyRhs && b + 32 + lane < hi) ? __ldcs(a.idx + b + 32 + lane) : 0;
       const int cnt = (int)(hi - b < 32 ? hi - b : 32);
       for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
-        float x[kEdges][kTiles], y[kEdges][kTiles];
+        float x[kEdges][NV], y[kEdges][NV];
 #pragma unroll
         for (int i = 0; i < kEdges; ++i) {
           const int e = e0 + i * NG + grp;
           const int32_t u = __shfl_sync(kAll, my_u, e & 31);
           const float* xrow = BIN != kCopyRhs ? a.X + (size_t)u * F : nullptr;
           const float* yrow = BIN != kCopyLhs ? a.Y + (size_t)(e < cnt ? b + e : b) * cols : nullptr;
+          float y1 = 1.f;
+          if (BIN != kCopyLhs && cols == 1) y1 = __ldg(yrow);
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            x[i][t] = BIN != kCopyRhs ? __ldg(xrow + j[t]) : 0.f;
-            y[i][t] = BIN != kCopyLhs ? __ldg(yrow + (cols == 1 ? 0 : j[t])) : 1.f;
+          for (int t = 0; t < kT; ++t) {
+            if (!tile_on[t]) continue;
+            if (VEC == 2) {
+              float2 xv = make_float2(0.f, 0.f), yv = make_float2(y1, y1);
+              if (BIN != kCopyRhs) xv = __ldg(reinterpret_cast<const float2*>(xrow + base[t]));
+              if (BIN != kCopyLhs && cols != 1)
+                yv = __ldg(reinterpret_cast<const float2*>(yrow + base[t]));
+              x[i][t * 2 + 0] = xv.x; x[i][t * 2 + 1] = xv.y;
+              y[i][t * 2 + 0] = yv.x; y[i][t * 2 + 1] = yv.y;
+            } else if (VEC == 4) {
+              float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), yv = make_float4(y1, y1, y1, y1);
+              if (BIN != kCopyRhs) xv = __ldg(reinterpret_cast<const float4*>(xrow + base[t]));
+              if (BIN != kCopyLhs && cols != 1)
+                yv = __ldg(reinterpret_cast<const float4*>(yrow + base[t]));
+              x[i][t * 4 + 0] = xv.x; x[i][t * 4 + 1] = xv.y;
+              x[i][t * 4 + 2] = xv.z; x[i][t * 4 + 3] = xv.w;
+              y[i][t * 4 + 0] = yv.x; y[i][t * 4 + 1] = yv.y;
+              y[i][t * 4 + 2] = yv.z; y[i][t * 4 + 3] = yv.w;
+            } else {
+              x[i][t] = BIN != kCopyRhs ? __ldg(xrow + base[t]) : 0.f;
+              y[i][t] = (BIN != kCopyLhs && cols != 1) ? __ldg(yrow + base[t]) : y1;
+            }
           }
         }
 #pragma unroll
@@ -141,17 +173,18 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
           const int e = e0 + i * NG + grp;
           const bool valid = e < cnt;
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            const float m = message<BIN>(x[i][t], y[i][t]);
+          for (int q = 0; q < NV; ++q) {
+            if (!tile_on[q / VEC]) continue;
+            const float m = message<BIN>(x[i][q], y[i][q]);
             if (RED == kSum) {
-              acc[t] += valid ? m : 0.f;
+              acc[q] += valid ? m : 0.f;
             } else {
               // a lane meets its edges in ascending position, so "strictly better" keeps the
               // lowest position among equal messages; lane groups are merged by take_better
               const bool take =
-                  valid && (best_k[t] < 0 || (RED == kMax ? m > best[t] : m < best[t]));
-              best[t] = take ? m : best[t];
-              best_k[t] = take ? (int32_t)(b + e) : best_k[t];
+                  valid && (best_k[q] < 0 || (RED == kMax ? m > best[q] : m < best[q]));
+              best[q] = take ? m : best[q];
+              best_k[q] = take ? (int32_t)(b + e) : best_k[q];
             }
           }
         }
@@ -159,29 +192,30 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
         if (RED == kSum && chain >= kChain) {
           chain = 0;
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) { total[t] += acc[t]; acc[t] = 0.f; }
+          for (int q = 0; q < NV; ++q) { total[q] += acc[q]; acc[q] = 0.f; }
         }
       }
     }
 #pragma unroll
-    for (int t = 0; t < kTiles; ++t) {
-      total[t] += acc[t];
+    for (int q = 0; q < NV; ++q) {
+      if (!tile_on[q / VEC]) continue;
+      total[q] += acc[q];
       for (int off = G; off < 32; off <<= 1) {
         if (RED == kSum) {
-          total[t] += __shfl_xor_sync(kAll, total[t], off);
+          total[q] += __shfl_xor_sync(kAll, total[q], off);
         } else {
-          const float ob = __shfl_xor_sync(kAll, best[t], off);
-          const int32_t ok = __shfl_xor_sync(kAll, best_k[t], off);
-          take_better<RED>(best[t], best_k[t], ob, ok);
+          const float ob = __shfl_xor_sync(kAll, best[q], off);
+          const int32_t ok2 = __shfl_xor_sync(kAll, best_k[q], off);
+          take_better<RED>(best[q], best_k[q], ob, ok2);
         }
       }
-      if (grp == 0 && jok[t]) {
-        const size_t o = (size_t)row * F + j[t];
+      if (grp == 0 && ok[q / VEC]) {
+        const size_t o = (size_t)row * F + base[q / VEC] + q % VEC;
         if (RED == kSum) {
-          a.out[o] = total[t];
+          a.out[o] = total[q];
         } else {
-          a.out[o] = best_k[t] >= 0 ? best[t] : 0.f;
-          if (a.arg_out) a.arg_out[o] = best_k[t];
+          a.out[o] = best_k[q] >= 0 ? best[q] : 0.f;
+          if (a.arg_out) a.arg_out[o] = best_k[q];
         }
       }
     }
@@ -520,7 +554,17 @@ dg_status_t dispatch_ops(int bin, int red, const GenArgs& a, cudaStream_t s) {
       return DG_OK;                                                           \
     }                                                                         \
   };
-DG_GEN_LAUNCHER(FwdLauncher, general_fwd_kernel)
+template <int BIN, int RED>
+struct FwdLauncher {
+  static dg_status_t run(const GenArgs& a, cudaStream_t s) {
+    if (a.vec == 4) general_fwd_kernel<BIN, RED, 4><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    else if (a.vec == 2) general_fwd_kernel<BIN, RED, 2><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    else general_fwd_kernel<BIN, RED, 1><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    DG_CUDA(cudaGetLastError());
+    count_launches(1);
+    return DG_OK;
+  }
+};
 DG_GEN_LAUNCHER(BwdVertexLauncher, general_bwd_vertex_kernel)
 DG_GEN_LAUNCHER(BwdEdgeFullLauncher, general_bwd_edge_full_kernel)
 DG_GEN_LAUNCHER(BwdEdgeScalarLauncher, general_bwd_edge_scalar_kernel)
@@ -572,7 +616,11 @@ dg_status_t dg_ap_fwd(dg_graph_t g, const float* fV, const float* fE, int32_t fE
   a.n = g->n;
   a.F = F;
   a.cols = binary == DG_BIN_COPY_LHS ? 1 : fE_cols;
-  a.log_g = log_group(F);
+  uintptr_t both = 0;
+  if (binary != DG_BIN_COPY_RHS) both |= (uintptr_t)fV;
+  if (binary != DG_BIN_COPY_LHS && a.cols != 1) both |= (uintptr_t)fE;
+  a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
+  a.log_g = log_group(F / a.vec);
   return dispatch_ops<FwdLauncher>((int)binary, (int)reduce, a, (cudaStream_t)stream);
 }
 
