@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(_ROOT, "include")
 LIB_PATH = os.path.join(_HERE, "libdgagg.so")
-SOURCES = ["dg_api.cu", "dg_graph.cu", "dg_transpose.cu", "dg_aggregate.cu", "dg_aggregate_self.cu",
+SOURCES = ["dg_api.cu", "dg_graph.cu", "dg_transpose.cu", "dg_aggregate.cu", "dg_aggregate_fold.cu", "dg_aggregate_self.cu", "dg_aggregate_self_fold.cu",
            "dg_static.cu", "dg_probe.cu", "dg_general.cu", "dg_reorder.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math=false"]

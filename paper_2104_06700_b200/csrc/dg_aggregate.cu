@@ -1,13 +1,15 @@
 // Host side of the aggregation: chooses the launch shape of one call (vector width, feature
 // slices, source blocks) and runs one launch per source block.  The kernels are in
-// dg_aggregate_kernels.cuh; this file compiles them for graphs without implicit self loops,
-// dg_aggregate_self.cu for graphs with them.
+// dg_aggregate_kernels.cuh; this file compiles them for graphs without implicit self loops and
+// without long segments, dg_aggregate_fold.cu, dg_aggregate_self.cu and dg_aggregate_self_fold.cu
+// for the other three combinations (four translation units compile side by side).
 #include "dg_aggregate_kernels.cuh"
 
 namespace dg {
 
 dg_status_t launch_plain(const Graph* g, const ApArgs& a, int vec, int slices, cudaStream_t s) {
-  return dispatch_type<false>(g, a, SelfArgs{}, vec, slices, s);
+  if (a.long_segments) return launch_plain_fold(g, a, vec, slices, s);
+  return dispatch_type<false, false>(g, a, SelfArgs{}, vec, slices, s);
 }
 
 // Bytes of L2 one row slice of `slice` elements of `eb` bytes occupies: L2 allocates 128-byte

@@ -665,9 +665,15 @@ dg_status_t launch_variant(const Graph* g, const ApArgs& a, const SelfArgs& sa, 
   constexpr bool kCapped = (SCALED && VEC * CPL * E::kBytes <= 16 && G >= 16) || G <= 4;
   const int64_t rows_per_block = (int64_t)a.rows_per_warp * kWarpsPerBlock;
   const int64_t light_blocks = (a.n + rows_per_block - 1) / rows_per_block;
+  // Where the cap pays depends on the graph as well: with rows sorted hub-first, or very short
+  // rows whose gathers come from DRAM, the scaled kernels run faster at their natural 60 registers
+  // (Products-like hub-first, mean backward: 6.02 -> 5.43 ms; Papers-like x0.1, mean backward:
+  // 13.9 -> 12.3 ms), while the same graph as generated and the dense-ish ones lose 8-15 % without
+  // it.  The handle says which (a.full_registers); the narrowest slices always keep the cap.
+  const bool capped = kCapped && (G <= 4 || !a.full_registers);
   if constexpr (SELF) {
     void (*kernel)(const ApArgs, const int, const SelfArgs);
-    if constexpr (kCapped) {
+    if (capped) {
       kernel = a.seg_lo ? ap_kernel_self_r40<E, VEC, G, CPL, SCALED, true, FOLD>
                         : ap_kernel_self_r40<E, VEC, G, CPL, SCALED, false, FOLD>;
     } else {
@@ -679,7 +685,7 @@ dg_status_t launch_variant(const Graph* g, const ApArgs& a, const SelfArgs& sa, 
     kernel<<<grid, kBlock, 0, s>>>(a, heavy_blocks, sa);
   } else {
     void (*kernel)(const ApArgs, const int);
-    if constexpr (kCapped) {
+    if (capped) {
       kernel = a.seg_lo ? ap_kernel_r40<E, VEC, G, CPL, SCALED, true, FOLD>
                         : ap_kernel_r40<E, VEC, G, CPL, SCALED, false, FOLD>;
     } else {
@@ -695,47 +701,41 @@ dg_status_t launch_variant(const Graph* g, const ApArgs& a, const SelfArgs& sa, 
   return DG_OK;
 }
 
-template <typename E, int VEC, int G, int CPL, bool SCALED, bool SELF>
-dg_status_t launch_pair(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
-                        cudaStream_t s) {
-  if (a.n == 0) return DG_OK;
-  return a.long_segments ? launch_variant<E, VEC, G, CPL, SCALED, SELF, true>(g, a, sa, slices, s)
-                         : launch_variant<E, VEC, G, CPL, SCALED, SELF, false>(g, a, sa, slices, s);
-}
-
-template <typename E, int VEC, bool SCALED, bool SELF>
+template <typename E, int VEC, bool SCALED, bool SELF, bool FOLD>
 dg_status_t dispatch_shape(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
                            cudaStream_t s) {
+  if (a.n == 0) return DG_OK;
   const int chunks = (a.slice_f < a.F ? a.slice_f : a.F) / VEC;  // vectors per row slice
-  if (chunks <= 2) return launch_pair<E, VEC, 2, 1, SCALED, SELF>(g, a, sa, slices, s);
-  if (chunks <= 4) return launch_pair<E, VEC, 4, 1, SCALED, SELF>(g, a, sa, slices, s);
-  if (chunks <= 8) return launch_pair<E, VEC, 8, 1, SCALED, SELF>(g, a, sa, slices, s);
-  if (chunks <= 16) return launch_pair<E, VEC, 16, 1, SCALED, SELF>(g, a, sa, slices, s);
-  if (chunks <= 32) return launch_pair<E, VEC, 32, 1, SCALED, SELF>(g, a, sa, slices, s);
-  if (chunks <= 64) return launch_pair<E, VEC, 32, 2, SCALED, SELF>(g, a, sa, slices, s);
-  return launch_pair<E, VEC, 32, 4, SCALED, SELF>(g, a, sa, slices, s);
+  if (chunks <= 2) return launch_variant<E, VEC, 2, 1, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  if (chunks <= 4) return launch_variant<E, VEC, 4, 1, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  if (chunks <= 8) return launch_variant<E, VEC, 8, 1, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  if (chunks <= 16) return launch_variant<E, VEC, 16, 1, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  if (chunks <= 32) return launch_variant<E, VEC, 32, 1, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  if (chunks <= 64) return launch_variant<E, VEC, 32, 2, SCALED, SELF, FOLD>(g, a, sa, slices, s);
+  return launch_variant<E, VEC, 32, 4, SCALED, SELF, FOLD>(g, a, sa, slices, s);
 }
 
-template <typename E, int VEC, bool SELF>
+template <typename E, int VEC, bool SELF, bool FOLD>
 dg_status_t dispatch_scaled(const Graph* g, const ApArgs& a, const SelfArgs& sa, int slices,
                             cudaStream_t s) {
-  return a.w ? dispatch_shape<E, VEC, true, SELF>(g, a, sa, slices, s)
-             : dispatch_shape<E, VEC, false, SELF>(g, a, sa, slices, s);
+  return a.w ? dispatch_shape<E, VEC, true, SELF, FOLD>(g, a, sa, slices, s)
+             : dispatch_shape<E, VEC, false, SELF, FOLD>(g, a, sa, slices, s);
 }
 
 // Storage type and vector width chosen by the caller; SELF = the graph has implicit self loops
-// (sa.self_ptr is set).  The two values of SELF are compiled in separate translation units.
-template <bool SELF>
+// (sa.self_ptr is set); FOLD = the graph may hold segments of kLongSegment entries or more in this
+// direction.  The four (SELF, FOLD) combinations are compiled in translation units of their own.
+template <bool SELF, bool FOLD>
 dg_status_t dispatch_type(const Graph* g, const ApArgs& a, const SelfArgs& sa, int vec, int slices,
                           cudaStream_t s) {
   if (a.x_bf16) {
-    if (vec == 8) return dispatch_scaled<BF16, 8, SELF>(g, a, sa, slices, s);
-    if (vec == 4) return dispatch_scaled<BF16, 4, SELF>(g, a, sa, slices, s);
-    return dispatch_scaled<BF16, 2, SELF>(g, a, sa, slices, s);
+    if (vec == 8) return dispatch_scaled<BF16, 8, SELF, FOLD>(g, a, sa, slices, s);
+    if (vec == 4) return dispatch_scaled<BF16, 4, SELF, FOLD>(g, a, sa, slices, s);
+    return dispatch_scaled<BF16, 2, SELF, FOLD>(g, a, sa, slices, s);
   }
-  if (vec == 4) return dispatch_scaled<F32, 4, SELF>(g, a, sa, slices, s);
-  if (vec == 2) return dispatch_scaled<F32, 2, SELF>(g, a, sa, slices, s);
-  return dispatch_scaled<F32, 1, SELF>(g, a, sa, slices, s);
+  if (vec == 4) return dispatch_scaled<F32, 4, SELF, FOLD>(g, a, sa, slices, s);
+  if (vec == 2) return dispatch_scaled<F32, 2, SELF, FOLD>(g, a, sa, slices, s);
+  return dispatch_scaled<F32, 1, SELF, FOLD>(g, a, sa, slices, s);
 }
 
 }  // namespace

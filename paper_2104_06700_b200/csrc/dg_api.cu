@@ -100,6 +100,12 @@ static dg_status_t count_long_rows(Graph* g) {
   return DG_OK;
 }
 
+// Graphs on which the scaled kernels run better without their register cap: renamed hub-first,
+// or fewer than 32 edges per vertex (see launch_variant).
+static int full_registers(const Graph* g) {
+  return g->degree_ordered || (g->n > 0 && g->nnz < 32 * g->n);
+}
+
 static int long_columns(Graph* g) {
   if (g->long_cols < 0 && cudaEventQuery(g->long_cols_ready) == cudaSuccess)
     g->long_cols = *g->long_cols_host > 0 ? 1 : 0;
@@ -163,6 +169,7 @@ static dg_status_t run_forward(Graph* g, const void* H, bool bf16, int32_t F, dg
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
   a.long_segments = g->long_rows;
+  a.full_registers = full_registers(g);
   const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
   return aggregate_run(g, a, sa, g->split_csr, (cudaStream_t)stream);
 }
@@ -194,6 +201,7 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   a.heavy_threshold = (int32_t)g->heavy_threshold;
   a.rows_per_warp = rows_per_warp(g);
   a.long_segments = long_columns(g);
+  a.full_registers = full_registers(g);
   const SelfArgs sa{g->self_loops ? g->rowptr : nullptr, op == DG_OP_MEAN};
   return aggregate_run(g, a, sa, g->split_csc, (cudaStream_t)stream);
 }

@@ -479,7 +479,8 @@ __device__ __forceinline__ void edge_grad_row(const EdgeGradArgs& a, int64_t v, 
 }
 
 template <int VEC, int G>
-__global__ void __launch_bounds__(kGenBlock) edge_grad_kernel(const EdgeGradArgs a,
+// four blocks per SM (64 registers): Products-like F = 100 10.9 -> 9.2 ms against the compiler's 74
+__global__ void __launch_bounds__(kGenBlock, 4) edge_grad_kernel(const EdgeGradArgs a,
                                                               const int heavy_blocks) {
   const int warp = threadIdx.x >> 5;
   if ((int)blockIdx.x < heavy_blocks) {

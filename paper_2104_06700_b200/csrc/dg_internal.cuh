@@ -54,6 +54,7 @@ struct dg_graph {
   // set on a handle made by dg_graph_reorder: arrays inside the caller's reorder storage
   const int32_t* new_of_old = nullptr;   // n: new id of every old vertex
   const int32_t* reorder_pos = nullptr;  // nnz: old CSR position of every new position
+  bool degree_ordered = false;           // made by dg_graph_reorder with a hub-first order
 
   int device = 0;
   int sm_count = 148;
@@ -97,6 +98,7 @@ struct ApArgs {
   const int32_t* seg_hi;      //   segment's piece (n entries each); nullptr = whole segments
   int32_t accumulate;         // source-blocked pass after the first: add to what Y holds
   int32_t long_segments;      // host side only: a segment of 2^15 entries or more may exist
+  int32_t full_registers;     // host side only: run the scaled kernels without the register cap
 };
 
 // Implicit self loops (every vertex its own neighbour with weight 1): row r also receives
@@ -115,6 +117,11 @@ struct SelfArgs {
 dg_status_t launch_plain(const dg_graph* g, const ApArgs& a, int vec, int slices, cudaStream_t s);
 dg_status_t launch_with_self_loops(const dg_graph* g, const ApArgs& a, const SelfArgs& sa, int vec,
                                    int slices, cudaStream_t s);
+// the same with the two-level sum for long segments (dg_aggregate_fold.cu, dg_aggregate_self_fold.cu)
+dg_status_t launch_plain_fold(const dg_graph* g, const ApArgs& a, int vec, int slices,
+                              cudaStream_t s);
+dg_status_t launch_with_self_loops_fold(const dg_graph* g, const ApArgs& a, const SelfArgs& sa,
+                                        int vec, int slices, cudaStream_t s);
 
 // Records the calling thread's last error message (printf-style, truncated to a fixed buffer:
 // nothing on an error path allocates, so nothing can throw across the C boundary).

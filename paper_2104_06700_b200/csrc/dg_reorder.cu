@@ -248,6 +248,7 @@ dg_status_t dg_graph_reorder(dg_graph_t g, dg_order_t order, const int32_t* give
   h->new_of_old = new_of_old;
   h->reorder_pos = reinterpret_cast<const int32_t*>(pos2);
   h->self_loops = g->self_loops;
+  h->degree_ordered = order != DG_ORDER_GIVEN;
   *out_graph = h;
   return DG_OK;
 }
