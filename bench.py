@@ -530,6 +530,24 @@ def extra_records(torch, binding, synth, name, g, sg, F, n_ref, peak, flush):
                                              fO=fO, arg=arg), 10, fl)
     out.append(rec("dg_ap_fwd (copylhs, max) + arg", ms,
                    idx_bytes + n_ref * F * 4 + 2 * sg.n * F * 4, "element-wise max with arg indices"))
+    if g.dg_graph_get_param("self_loops") == 0:
+        try:
+            g.dg_graph_get_csc()
+            have_csc = True
+        except binding.DgError:
+            have_csc = False
+        if have_csc:
+            dV = torch.empty_like(H)
+            bwd = lambda: binding._check(binding.lib().dg_ap_bwd(
+                g._h, G.data_ptr(), H.data_ptr(), None, 1, F, binding.DG_BIN_COPY_LHS,
+                binding.DG_RED_MAX, arg.data_ptr(), dV.data_ptr(), None,
+                torch.cuda.current_stream().cuda_stream))
+            ms = time_one(torch, bwd, 10, fl)
+            out.append(rec("dg_ap_bwd (copylhs, max): dV", ms,
+                           idx_bytes + sg.nnz * 4 + 3 * sg.n * F * 4,
+                           "gather over the CSC with an equality test on arg (dO and arg rows per "
+                           "edge), no atomics"))
+            del dV
     del arg
     if sg.nnz * F * 4 <= 24e9:
         fE = torch.rand((sg.nnz, F), device=dev, dtype=torch.float32)
@@ -622,7 +640,8 @@ def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_
                 b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False)
                 b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_nonempty, op == "mean")
                 rec = {"workload": name, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
-                       "weighted": weighted, "reorder": reorder or "none", "reps": reps,
+                       "weighted": weighted, "reorder": reorder or "none", "dtype": "f32",
+                       "reps": reps,
                        "l2": "flushed before every call (inputs fit L2)" if cold
                              else "inputs larger than L2 (no flush needed)",
                        "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
@@ -635,6 +654,40 @@ def run_workloads(torch, binding, synth, dev, device_index, peak, ceilings, cpu_
                 rec["cpu_baseline"] = None if cpu_seconds <= 0 else cpu_baseline_sampled(
                     torch, sg, (colptr, rowidx_T, w_T), H, G, op, cpu_seconds)
                 records.append(rec)
+            # the gathered matrices stored as bf16 (sums and outputs fp32): the two largest graphs
+            if (name, F, reorder) in (("products_like", 100, None), ("papers_like", 128, None)):
+                if two_buffers:
+                    # no room for a third matrix: the bf16 copy is packed into H's own storage,
+                    # chunk by chunk from the front (H is not needed as fp32 after this point)
+                    flat16 = H.view(-1).view(torch.bfloat16)
+                    rows = max(1, (1 << 28) // F)
+                    for s0 in range(0, sg.n, rows):
+                        e0 = min(sg.n, s0 + rows)
+                        tmp = H[s0:e0].to(torch.bfloat16)
+                        flat16[s0 * F:e0 * F] = tmp.view(-1)
+                        del tmp
+                    Hb = flat16[:sg.n * F].view(sg.n, F)
+                else:
+                    Hb = H.to(torch.bfloat16)
+                Gb = Hb if two_buffers else G.to(torch.bfloat16)
+                for op in ops:
+                    code = binding.DG_OP_MEAN if op == "mean" else binding.DG_OP_SUM
+                    fwd_call = lambda: g.dg_aggregate_fwd_bf16(Hb, code, out=out)
+                    bwd_call = lambda: g.dg_aggregate_bwd_bf16(Gb, code, dH=dH)
+                    f_ms, b_ms, clocks = time_calls(torch, fwd_call, bwd_call, 5 if mat_bytes > 1e10 else 10,
+                                                    None, device_index)
+                    b_fwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_ref, False, 2)
+                    b_bwd = compulsory_bytes(sg.n, sg.nnz, F, weighted, n_nonempty, op == "mean", 2)
+                    records.append({
+                        "workload": name, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
+                        "weighted": weighted, "reorder": "none",
+                        "dtype": "f32 sums over bf16-stored inputs (not the fp32 headline)",
+                        "reps": len(f_ms), "l2": "inputs larger than L2 (no flush needed)",
+                        "fwd": direction_record(f_ms, b_fwd, sg.nnz * F * 2, sg.nnz * F, peak, None),
+                        "bwd": direction_record(b_ms, b_bwd, sg.nnz * F * 2, sg.nnz * F, peak, None),
+                        "traffic": {"fwd": None, "bwd": None}, "clocks": clocks,
+                        "cpu_baseline": None})
+                del Hb, Gb
             if dims and F == dims[0]:
                 epochs[label] = epoch_plain(torch, g, sg, H, dims, frac, dev)
             del H, out, G, dH
@@ -1031,7 +1084,7 @@ def main():
                    and args.reorder == "none")
     if rank == 0 and world == 1 and args.workloads == "all" and default_run:
         head = {"workload": args.workload, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
-                "weighted": weighted, "reorder": "none", "reps": args.steps,
+                "weighted": weighted, "reorder": "none", "dtype": "f32", "reps": args.steps,
                 "l2": "inputs larger than L2 (no flush needed)",
                 "buffers": "H, out, dOut, dH separate",
                 "fwd": direction_record(fwd_list, b_fwd, sg.nnz * F * 4, sg.nnz * F, peak, ceilings),

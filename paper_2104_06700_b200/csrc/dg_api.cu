@@ -107,8 +107,12 @@ static int full_registers(const Graph* g) {
 }
 
 static int long_columns(Graph* g) {
-  if (g->long_cols < 0 && cudaEventQuery(g->long_cols_ready) == cudaSuccess)
-    g->long_cols = *g->long_cols_host > 0 ? 1 : 0;
+  if (g->long_cols < 0) {
+    if (cudaEventQuery(g->long_cols_ready) == cudaSuccess)
+      g->long_cols = *g->long_cols_host > 0 ? 1 : 0;
+    else
+      (void)cudaGetLastError();  // "not ready" must not be mistaken for a failed launch later
+  }
   return g->long_cols != 0;
 }
 

@@ -44,7 +44,7 @@ struct GenArgs {
   int32_t F, cols;
   int32_t log_g;         // lanes per edge = 1 << log_g
   int32_t row_scale;     // edge-weight gradient: 0 none, 1 = 1/deg(v), 2 = 1/(deg(v)+1)
-  int32_t vec;           // forward: floats per load, 4 or 2 when F and the operands' alignment allow
+  int32_t vec;           // floats per load, 4 or 2 when F and the operands' alignment allow
 };
 
 // one fp32 IEEE operation, never contracted into a neighbouring add
@@ -225,9 +225,13 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
 // Gradient with respect to fV: warp per source vertex u over its CSC segment,
 //   dV[u][j] = sum_q sel * dO[v_q][j] * d(x (x) y)/dx,   sel = [arg[v_q][j] == perm[q]] (max/min)
 // The derivative depends on y only (and not at all for copylhs / add / sub).  Same walk as the
-// forward kernel: batched indices (destination and CSR position), unpredicated loads.
-template <int BIN, int RED>
+// forward kernel: batched indices (destination and CSR position), four values per lane and edge
+// in vectors of VEC floats, unpredicated loads.
+template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const GenArgs a) {
+  constexpr int kT = kTiles / VEC;
+  constexpr int NV = kT * VEC;
+  constexpr int kEdges = 2;
   const int lane = threadIdx.x & 31;
   const int64_t u = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
   if (u >= a.n) return;
@@ -237,17 +241,18 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
   const int F = a.F, cols = a.cols;
   constexpr bool kNeedsY = BIN == kMul || BIN == kDiv;
   constexpr bool kNeedsK = kNeedsY || RED != kSum;
-  constexpr int kEdges = 2;
-  for (int f0 = 0; f0 < F; f0 += kTiles * G) {
-    bool jok[kTiles];
-    int j[kTiles];
-    float acc[kTiles], total[kTiles];
+  for (int f0 = 0; f0 < F; f0 += kT * G * VEC) {
+    bool ok[kT], tile_on[kT];
+    int base[kT];
+    float acc[NV], total[NV];
 #pragma unroll
-    for (int t = 0; t < kTiles; ++t) {
-      jok[t] = f0 + t * G + c < F;
-      j[t] = jok[t] ? f0 + t * G + c : 0;
-      acc[t] = total[t] = 0.f;
+    for (int t = 0; t < kT; ++t) {
+      tile_on[t] = f0 + t * G * VEC < F;
+      ok[t] = f0 + (t * G + c) * VEC < F;
+      base[t] = ok[t] ? f0 + (t * G + c) * VEC : 0;
     }
+#pragma unroll
+    for (int q = 0; q < NV; ++q) acc[q] = total[q] = 0.f;
     int chain = 0;
     for (int64_t b = lo; b < hi; b += 32) {
       const bool mine = b + lane < hi;
@@ -255,44 +260,70 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
       const int32_t my_k = (kNeedsK && mine) ? __ldcs(a.perm + b + lane) : 0;
       const int cnt = (int)(hi - b < 32 ? hi - b : 32);
       for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
-        float g[kEdges][kTiles], y[kEdges][kTiles];
-        int32_t sel[kEdges][kTiles], k[kEdges];
+        float g[kEdges][NV], y[kEdges][NV];
+        int32_t sel[kEdges][NV], k[kEdges];
 #pragma unroll
         for (int i = 0; i < kEdges; ++i) {
           const int e = e0 + i * NG + grp;
           const size_t vrow = (size_t)__shfl_sync(kAll, my_v, e & 31) * F;
           k[i] = __shfl_sync(kAll, my_k, e & 31);
+          const float* yrow = kNeedsY ? a.Y + (size_t)k[i] * cols : nullptr;
+          float y1 = 1.f;
+          if (kNeedsY && cols == 1) y1 = __ldg(yrow);
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            g[i][t] = __ldg(a.X + vrow + j[t]);  // dO[v][j]
-            y[i][t] = kNeedsY ? __ldg(a.Y + (size_t)k[i] * cols + (cols == 1 ? 0 : j[t])) : 1.f;
-            sel[i][t] = RED != kSum ? __ldg(a.arg + vrow + j[t]) : 0;
+          for (int t = 0; t < kT; ++t) {
+            if (!tile_on[t]) continue;
+            if (VEC == 4) {
+              const float4 gv = __ldg(reinterpret_cast<const float4*>(a.X + vrow + base[t]));
+              float4 yv = make_float4(y1, y1, y1, y1);
+              int4 sv = make_int4(0, 0, 0, 0);
+              if (kNeedsY && cols != 1) yv = __ldg(reinterpret_cast<const float4*>(yrow + base[t]));
+              if (RED != kSum) sv = __ldg(reinterpret_cast<const int4*>(a.arg + vrow + base[t]));
+              g[i][t * 4 + 0] = gv.x; g[i][t * 4 + 1] = gv.y; g[i][t * 4 + 2] = gv.z; g[i][t * 4 + 3] = gv.w;
+              y[i][t * 4 + 0] = yv.x; y[i][t * 4 + 1] = yv.y; y[i][t * 4 + 2] = yv.z; y[i][t * 4 + 3] = yv.w;
+              sel[i][t * 4 + 0] = sv.x; sel[i][t * 4 + 1] = sv.y; sel[i][t * 4 + 2] = sv.z; sel[i][t * 4 + 3] = sv.w;
+            } else if (VEC == 2) {
+              const float2 gv = __ldg(reinterpret_cast<const float2*>(a.X + vrow + base[t]));
+              float2 yv = make_float2(y1, y1);
+              int2 sv = make_int2(0, 0);
+              if (kNeedsY && cols != 1) yv = __ldg(reinterpret_cast<const float2*>(yrow + base[t]));
+              if (RED != kSum) sv = __ldg(reinterpret_cast<const int2*>(a.arg + vrow + base[t]));
+              g[i][t * 2 + 0] = gv.x; g[i][t * 2 + 1] = gv.y;
+              y[i][t * 2 + 0] = yv.x; y[i][t * 2 + 1] = yv.y;
+              sel[i][t * 2 + 0] = sv.x; sel[i][t * 2 + 1] = sv.y;
+            } else {
+              g[i][t] = __ldg(a.X + vrow + base[t]);
+              y[i][t] = (kNeedsY && cols != 1) ? __ldg(yrow + base[t]) : y1;
+              sel[i][t] = RED != kSum ? __ldg(a.arg + vrow + base[t]) : 0;
+            }
           }
         }
 #pragma unroll
         for (int i = 0; i < kEdges; ++i) {
           const bool valid = e0 + i * NG + grp < cnt;
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) {
-            float v = g[i][t];
-            if (kNeedsY) v *= d_dx<BIN>(y[i][t]);
-            if (!valid || (RED != kSum && sel[i][t] != k[i])) v = 0.f;
-            acc[t] += v;
+          for (int q = 0; q < NV; ++q) {
+            if (!tile_on[q / VEC]) continue;
+            float v = g[i][q];
+            if (kNeedsY) v *= d_dx<BIN>(y[i][q]);
+            if (!valid || (RED != kSum && sel[i][q] != k[i])) v = 0.f;
+            acc[q] += v;
           }
         }
         chain += kEdges;
         if (chain >= kChain) {
           chain = 0;
 #pragma unroll
-          for (int t = 0; t < kTiles; ++t) { total[t] += acc[t]; acc[t] = 0.f; }
+          for (int q = 0; q < NV; ++q) { total[q] += acc[q]; acc[q] = 0.f; }
         }
       }
     }
 #pragma unroll
-    for (int t = 0; t < kTiles; ++t) {
-      total[t] += acc[t];
-      for (int off = G; off < 32; off <<= 1) total[t] += __shfl_xor_sync(kAll, total[t], off);
-      if (grp == 0 && jok[t]) a.out[(size_t)u * F + j[t]] = total[t];
+    for (int q = 0; q < NV; ++q) {
+      if (!tile_on[q / VEC]) continue;
+      total[q] += acc[q];
+      for (int off = G; off < 32; off <<= 1) total[q] += __shfl_xor_sync(kAll, total[q], off);
+      if (grp == 0 && ok[q / VEC]) a.out[(size_t)u * F + base[q / VEC] + q % VEC] = total[q];
     }
   }
 }
@@ -566,7 +597,17 @@ struct FwdLauncher {
     return DG_OK;
   }
 };
-DG_GEN_LAUNCHER(BwdVertexLauncher, general_bwd_vertex_kernel)
+template <int BIN, int RED>
+struct BwdVertexLauncher {
+  static dg_status_t run(const GenArgs& a, cudaStream_t s) {
+    if (a.vec == 4) general_bwd_vertex_kernel<BIN, RED, 4><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    else if (a.vec == 2) general_bwd_vertex_kernel<BIN, RED, 2><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    else general_bwd_vertex_kernel<BIN, RED, 1><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    DG_CUDA(cudaGetLastError());
+    count_launches(1);
+    return DG_OK;
+  }
+};
 DG_GEN_LAUNCHER(BwdEdgeFullLauncher, general_bwd_edge_full_kernel)
 DG_GEN_LAUNCHER(BwdEdgeScalarLauncher, general_bwd_edge_scalar_kernel)
 #undef DG_GEN_LAUNCHER
@@ -654,7 +695,11 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
       a.n = g->n;
       a.F = F;
       a.cols = cols;
-      a.log_g = log_group(F);
+      uintptr_t both = (uintptr_t)dO;
+      if ((binary == DG_BIN_MUL || binary == DG_BIN_DIV) && cols != 1) both |= (uintptr_t)fE;
+      if (reduce != DG_RED_SUM) both |= (uintptr_t)arg;
+      a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
+      a.log_g = log_group(F / a.vec);
       if (dg_status_t st = dispatch_ops<BwdVertexLauncher>((int)binary, (int)reduce, a, s)) return st;
     }
   }

@@ -248,3 +248,36 @@ def test_papers_like_full_size():
                                   _pad_rows(to_np(H[uniq]), n_sub), oracle.OP_SUM,
                                   cols=np.arange(len(cols)))
     assert_within_bound(to_np(out[torch.as_tensor(cols, device=DEV)]), ref, mag, "bwd")
+
+
+def test_full_size_products_like_hub_first():
+    """dg_graph_reorder at the benchmark's size: the renamed CSR bit for bit against the oracle,
+    then forward and backward AP on the renamed handle (the launch configuration the bench times
+    for its hub-first records) against the oracle of the ORIGINAL graph, on every element."""
+    sg = synth.make("products_like", device=DEV)
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, sg.edge_w)
+    r = g.dg_graph_reorder(binding.DG_ORDER_OUT_DEGREE)
+    torch.cuda.synchronize()
+    rp, ci = to_np(sg.rowptr), to_np(sg.colidx)
+    order = oracle.order_by_degree(np.bincount(ci, minlength=sg.n).astype(np.int64))
+    assert np.array_equal(to_np(r.new_of_old), order), "new_of_old"
+    rp2, ci2, _, pos2 = oracle.relabel(rp, ci, None, order)
+    assert np.array_equal(to_np(r.rowptr), rp2), "rowptr"
+    assert np.array_equal(to_np(r.colidx), ci2), "colidx"
+    assert np.array_equal(to_np(r.pos).astype(np.int64), pos2), "pos"
+    del rp2, ci2, pos2
+    r.dg_graph_transpose()
+    colptr, rowidx_T, _, _ = oracle.transpose(rp, ci, None)
+    F = 100
+    H = synth.features(sg.n, F, 91, DEV)
+    G = synth.features(sg.n, F, 92, DEV)
+    H2 = binding.dg_permute_rows(r.new_of_old, H)
+    G2 = binding.dg_permute_rows(r.new_of_old, G)
+    for op in (binding.DG_OP_SUM, binding.DG_OP_MEAN):
+        out = binding.dg_permute_rows(r.new_of_old, r.dg_aggregate_fwd(H2, op), to_old=True)
+        dH = binding.dg_permute_rows(r.new_of_old, r.dg_aggregate_bwd(G2, op), to_old=True)
+        torch.cuda.synchronize()
+        ref, mag = oracle.ap_forward(rp, ci, None, to_np(H), op)
+        assert_within_bound(to_np(out), ref, mag, "fwd, hub-first")
+        ref, mag = oracle.ap_backward(rp, colptr, rowidx_T, None, to_np(G), op)
+        assert_within_bound(to_np(dH), ref, mag, "bwd, hub-first")
