@@ -138,6 +138,24 @@ def compulsory_bytes(n, nnz, F, weighted, n_ref, inv_deg_gather, in_bytes=4):
     return b
 
 
+def device_memory_bytes(torch):
+    if torch.cuda.is_available():
+        return torch.cuda.get_device_properties(torch.cuda.current_device()).total_memory
+    return 183e9
+
+
+def workload_config(args, sg, F, op, weighted, world, two_buffers):
+    """The `config` object of the JSON line: the same for both arms on the same workload."""
+    return {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz, "F": F,
+            "op": op, "weighted": weighted, "step": "fwd AP + bwd AP", "replicas": world,
+            "sorted_ids": bool(args.sorted_ids), "reorder": args.reorder,
+            "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
+                       else "H, out, dOut, dH separate",
+            "l2": "inputs larger than L2 (no flush needed)" if sg.n * F * 4 > 252e6
+                  else "inputs fit L2: warm-L2 numbers",
+            "knobs": args.set}
+
+
 def max_over_ranks(x: float, world: int, device="cpu") -> float:
     """Slowest rank's time: all-reduce(MAX) over the default process group (NCCL on GPUs, gloo in
     the CPU tests); the identity for one rank."""
@@ -263,8 +281,8 @@ def run_reference(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_sec / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
-                   "F": F, "op": op},
+        "config": workload_config(args, sg, F, op, w is not None, 1,
+                                  4 * sg.n * F * 4 > 0.6 * device_memory_bytes(torch)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
                          "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -1110,14 +1128,7 @@ def main():
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "f32" if not bf16 else "f32 sums over bf16-stored inputs", "data": "synthetic",
-            "config": {"workload": args.workload, "scale": args.scale, "n": sg.n, "nnz": sg.nnz,
-                       "F": F, "op": op, "weighted": weighted, "step": "fwd AP + bwd AP",
-                       "replicas": world, "sorted_ids": bool(args.sorted_ids),
-                       "reorder": args.reorder,
-                       "buffers": "H=dOut, out=dH (two n x F buffers)" if two_buffers
-                       else "H, out, dOut, dH separate", "l2": "inputs larger than L2 (no flush needed)"
-                       if sg.n * F * 4 > 252e6 else "inputs fit L2: warm-L2 numbers",
-                       "knobs": args.set},
+            "config": workload_config(args, sg, F, op, weighted, world, two_buffers),
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
             "clocks": clocks, "epoch": epoch_info,
             "ingest": {"graph_create_ms": create_ms, "transpose_ms": transpose_ms,
