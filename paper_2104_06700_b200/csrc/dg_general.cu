@@ -6,13 +6,14 @@
 // edges, Section 2.2).
 //
 // These kernels are kept apart from the sum / mean kernels of dg_aggregate_kernels.cuh, which
-// stay as they are: here a warp owns one row (one column in the pass over the CSC), its lanes
-// are spread along the features in groups of G lanes, and the groups take different edges.  With
+// stay as they are: here a warp owns one row (one column in the pass over the CSC; the 8 warps of
+// a block share a row of the handle's heavy list), its lanes are spread along the features in
+// groups of G lanes, and the groups take different edges.  With
 // a full edge-feature matrix the edge stream is as large as the gathered rows (nnz x F x 4
 // bytes, read once, coalesced), so these passes are bound by HBM streaming rather than by the
 // gather.
 //
-// Determinism: every output element is produced by one warp in a fixed order; the extremum of
+// Determinism: every output element is produced by one warp (one block) in a fixed order; the extremum of
 // max / min is chosen on (message, edge position) pairs, equal messages going to the lowest
 // position, so the order in which lane groups are combined does not matter.  No atomics.
 #include "dg_internal.cuh"
@@ -45,6 +46,12 @@ struct GenArgs {
   int32_t log_g;         // lanes per edge = 1 << log_g
   int32_t row_scale;     // edge-weight gradient: 0 none, 1 = 1/deg(v), 2 = 1/(deg(v)+1)
   int32_t vec;           // floats per load, 4 or 2 when F and the operands' alignment allow
+  // the handle's list of rows (columns, in the pass over the CSC) longer than heavy_threshold,
+  // longest first; nullptr: every row is walked by one warp
+  const int32_t* heavy_list;
+  const int32_t* heavy_count;
+  int32_t heavy_cap, heavy_threshold;
+  int32_t heavy_blocks;  // leading blocks of the grid that walk the heavy list
 };
 
 // one fp32 IEEE operation, never contracted into a neighbouring add
@@ -90,6 +97,286 @@ template <int BIN> struct EdgesInFlight {
   static constexpr int value = (BIN == kCopyLhs || BIN == kCopyRhs) ? 4 : 2;
 };
 
+// ---- rows on the handle's heavy list: a block per row ----
+//
+// The first heavy_blocks blocks of a launch walk the list (longest first); they start before the
+// blocks of the light rows, so a hub row runs beside the light ones instead of holding one warp
+// long after the rest of the grid has drained.  The 8 warps of a block take interleaved 32-edge
+// batches of one row, leave their partial results in shared memory, and warp 0 merges them in warp
+// order (sums) or by (message, position) (max / min), so the result does not depend on timing.
+// The walk below is the one of the light kernels with a batch stride; the light kernels keep it
+// written out in their bodies, which compiles to faster code than the call (Products-like max:
+// 13.0 against 21.0 ms).
+
+// where a lane's four values per edge lie: kTiles / VEC vectors of VEC floats, G * VEC apart
+template <int VEC>
+struct LaneTiles {
+  static constexpr int kT = kTiles / VEC;
+  bool ok[kT], tile_on[kT];
+  int base[kT];  // first feature of the lane's vector t (0 when it lies beyond F)
+  __device__ __forceinline__ void place(int f0, int F, int G, int c) {
+#pragma unroll
+    for (int t = 0; t < kT; ++t) {
+      tile_on[t] = f0 + t * G * VEC < F;  // the same for the whole warp
+      ok[t] = f0 + (t * G + c) * VEC < F;
+      base[t] = ok[t] ? f0 + (t * G + c) * VEC : 0;
+    }
+  }
+};
+
+// loads VEC consecutive floats (ints) into dst[0..VEC)
+template <int VEC>
+__device__ __forceinline__ void load_vec(float* dst, const float* src) {
+  if (VEC == 4) {
+    const float4 v = __ldg(reinterpret_cast<const float4*>(src));
+    dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+  } else if (VEC == 2) {
+    const float2 v = __ldg(reinterpret_cast<const float2*>(src));
+    dst[0] = v.x; dst[1] = v.y;
+  } else {
+    dst[0] = __ldg(src);
+  }
+}
+template <int VEC>
+__device__ __forceinline__ void load_vec(int32_t* dst, const int32_t* src) {
+  if (VEC == 4) {
+    const int4 v = __ldg(reinterpret_cast<const int4*>(src));
+    dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+  } else if (VEC == 2) {
+    const int2 v = __ldg(reinterpret_cast<const int2*>(src));
+    dst[0] = v.x; dst[1] = v.y;
+  } else {
+    dst[0] = __ldg(src);
+  }
+}
+
+// A warp's share of row [lo, hi): the 32-edge batches first_batch, first_batch + batch_stride, ...
+// Leaves the per-lane sums (total) or extrema (best, best_k; best_k < 0: none), not yet combined
+// across the lane groups.
+template <int BIN, int RED, int VEC>
+__device__ __forceinline__ void fwd_walk(const GenArgs& a, int64_t lo, int64_t hi, int first_batch,
+                                         int batch_stride, const LaneTiles<VEC>& L, int grp, int NG,
+                                         float (&total)[4], float (&best)[4], int32_t (&best_k)[4]) {
+  constexpr int kT = kTiles / VEC;
+  constexpr int kEdges = (VEC > 1 && EdgesInFlight<BIN>::value == 4) ? 4 : 2;
+  const int lane = threadIdx.x & 31;
+  const int F = a.F, cols = a.cols;
+  const int64_t step = (int64_t)batch_stride * 32;
+  float acc[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    acc[q] = total[q] = best[q] = 0.f;
+    best_k[q] = -1;
+  }
+  int chain = 0;
+  for (int64_t b = lo + (int64_t)first_batch * 32; b < hi; b += step) {
+    const int32_t my_u = (BIN != kCopyRhs && b + lane < hi) ? __ldcs(a.idx + b + lane) : 0;
+    const int cnt = (int)(hi - b < 32 ? hi - b : 32);
+    for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
+      float x[kEdges][4], y[kEdges][4];
+#pragma unroll
+      for (int i = 0; i < kEdges; ++i) {
+        const int e = e0 + i * NG + grp;
+        const int32_t u = __shfl_sync(kAll, my_u, e & 31);
+        const float* xrow = BIN != kCopyRhs ? a.X + (size_t)u * F : nullptr;
+        const float* yrow = BIN != kCopyLhs ? a.Y + (size_t)(e < cnt ? b + e : b) * cols : nullptr;
+        float y1 = 1.f;
+        if (BIN != kCopyLhs && cols == 1) y1 = __ldg(yrow);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { x[i][q] = 0.f; y[i][q] = y1; }
+#pragma unroll
+        for (int t = 0; t < kT; ++t) {
+          if (!L.tile_on[t]) continue;
+          if (BIN != kCopyRhs) load_vec<VEC>(&x[i][t * VEC], xrow + L.base[t]);
+          if (BIN != kCopyLhs && cols != 1) load_vec<VEC>(&y[i][t * VEC], yrow + L.base[t]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kEdges; ++i) {
+        const int e = e0 + i * NG + grp;
+        const bool valid = e < cnt;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (!L.tile_on[q / VEC]) continue;
+          const float m = message<BIN>(x[i][q], y[i][q]);
+          if (RED == kSum) {
+            acc[q] += valid ? m : 0.f;
+          } else {
+            // ascending positions within a lane: "strictly better" keeps the lowest among equals
+            const bool take =
+                valid && (best_k[q] < 0 || (RED == kMax ? m > best[q] : m < best[q]));
+            best[q] = take ? m : best[q];
+            best_k[q] = take ? (int32_t)(b + e) : best_k[q];
+          }
+        }
+      }
+      chain += kEdges;
+      if (RED == kSum && chain >= kChain) {
+        chain = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { total[q] += acc[q]; acc[q] = 0.f; }
+      }
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) total[q] += acc[q];
+}
+
+template <int BIN, int RED, int VEC>
+__device__ __forceinline__ void fwd_heavy_rows(const GenArgs& a, int first, int stride) {
+  __shared__ float part_v[kGenWarps][4][32];
+  __shared__ int32_t part_k[kGenWarps][4][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int G = 1 << a.log_g, NG = 32 >> a.log_g;
+  const int grp = lane >> a.log_g, c = lane & (G - 1);
+  const int count = min(*a.heavy_count, a.heavy_cap);
+  for (int i = first; i < count; i += stride) {
+    const int64_t row = a.heavy_list[i];
+    const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
+    for (int f0 = 0; f0 < a.F; f0 += kTiles * G) {
+      LaneTiles<VEC> L;
+      L.place(f0, a.F, G, c);
+      float total[4], best[4];
+      int32_t best_k[4];
+      fwd_walk<BIN, RED, VEC>(a, lo, hi, warp, kGenWarps, L, grp, NG, total, best, best_k);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        part_v[warp][q][lane] = RED == kSum ? total[q] : best[q];
+        part_k[warp][q][lane] = best_k[q];
+      }
+      __syncthreads();
+      if (warp == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (!L.tile_on[q / VEC]) continue;
+          for (int w = 1; w < kGenWarps; ++w) {
+            if (RED == kSum) total[q] += part_v[w][q][lane];
+            else take_better<RED>(best[q], best_k[q], part_v[w][q][lane], part_k[w][q][lane]);
+          }
+          for (int off = G; off < 32; off <<= 1) {
+            if (RED == kSum) {
+              total[q] += __shfl_xor_sync(kAll, total[q], off);
+            } else {
+              const float ob = __shfl_xor_sync(kAll, best[q], off);
+              const int32_t ok2 = __shfl_xor_sync(kAll, best_k[q], off);
+              take_better<RED>(best[q], best_k[q], ob, ok2);
+            }
+          }
+          if (grp == 0 && L.ok[q / VEC]) {
+            const size_t o = (size_t)row * a.F + L.base[q / VEC] + q % VEC;
+            if (RED == kSum) {
+              a.out[o] = total[q];
+            } else {
+              a.out[o] = best_k[q] >= 0 ? best[q] : 0.f;
+              if (a.arg_out) a.arg_out[o] = best_k[q];
+            }
+          }
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+// the same for a column of the CSC in the gradient with respect to fV
+template <int BIN, int RED, int VEC>
+__device__ __forceinline__ void bwd_walk(const GenArgs& a, int64_t lo, int64_t hi, int first_batch,
+                                         int batch_stride, const LaneTiles<VEC>& L, int grp, int NG,
+                                         float (&total)[4]) {
+  constexpr int kT = kTiles / VEC;
+  constexpr int kEdges = 2;
+  constexpr bool kNeedsY = BIN == kMul || BIN == kDiv;
+  constexpr bool kNeedsK = kNeedsY || RED != kSum;
+  const int lane = threadIdx.x & 31;
+  const int F = a.F, cols = a.cols;
+  const int64_t step = (int64_t)batch_stride * 32;
+  float acc[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) acc[q] = total[q] = 0.f;
+  int chain = 0;
+  for (int64_t b = lo + (int64_t)first_batch * 32; b < hi; b += step) {
+    const bool mine = b + lane < hi;
+    const int32_t my_v = mine ? __ldcs(a.idx + b + lane) : 0;
+    const int32_t my_k = (kNeedsK && mine) ? __ldcs(a.perm + b + lane) : 0;
+    const int cnt = (int)(hi - b < 32 ? hi - b : 32);
+    for (int e0 = 0; e0 < cnt; e0 += NG * kEdges) {
+      float g[kEdges][4], y[kEdges][4];
+      int32_t sel[kEdges][4], k[kEdges];
+#pragma unroll
+      for (int i = 0; i < kEdges; ++i) {
+        const int e = e0 + i * NG + grp;
+        const size_t vrow = (size_t)__shfl_sync(kAll, my_v, e & 31) * F;
+        k[i] = __shfl_sync(kAll, my_k, e & 31);
+        const float* yrow = kNeedsY ? a.Y + (size_t)k[i] * cols : nullptr;
+        float y1 = 1.f;
+        if (kNeedsY && cols == 1) y1 = __ldg(yrow);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { g[i][q] = 0.f; y[i][q] = y1; sel[i][q] = 0; }
+#pragma unroll
+        for (int t = 0; t < kT; ++t) {
+          if (!L.tile_on[t]) continue;
+          load_vec<VEC>(&g[i][t * VEC], a.X + vrow + L.base[t]);
+          if (kNeedsY && cols != 1) load_vec<VEC>(&y[i][t * VEC], yrow + L.base[t]);
+          if (RED != kSum) load_vec<VEC>(&sel[i][t * VEC], a.arg + vrow + L.base[t]);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kEdges; ++i) {
+        const bool valid = e0 + i * NG + grp < cnt;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (!L.tile_on[q / VEC]) continue;
+          float v = g[i][q];
+          if (kNeedsY) v *= d_dx<BIN>(y[i][q]);
+          if (!valid || (RED != kSum && sel[i][q] != k[i])) v = 0.f;
+          acc[q] += v;
+        }
+      }
+      chain += kEdges;
+      if (chain >= kChain) {
+        chain = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { total[q] += acc[q]; acc[q] = 0.f; }
+      }
+    }
+  }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) total[q] += acc[q];
+}
+
+template <int BIN, int RED, int VEC>
+__device__ __forceinline__ void bwd_heavy_cols(const GenArgs& a, int first, int stride) {
+  __shared__ float part_v[kGenWarps][4][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int G = 1 << a.log_g, NG = 32 >> a.log_g;
+  const int grp = lane >> a.log_g, c = lane & (G - 1);
+  const int count = min(*a.heavy_count, a.heavy_cap);
+  for (int i = first; i < count; i += stride) {
+    const int64_t u = a.heavy_list[i];
+    const int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
+    for (int f0 = 0; f0 < a.F; f0 += kTiles * G) {
+      LaneTiles<VEC> L;
+      L.place(f0, a.F, G, c);
+      float total[4];
+      bwd_walk<BIN, RED, VEC>(a, lo, hi, warp, kGenWarps, L, grp, NG, total);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) part_v[warp][q][lane] = total[q];
+      __syncthreads();
+      if (warp == 0) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (!L.tile_on[q / VEC]) continue;
+          for (int w = 1; w < kGenWarps; ++w) total[q] += part_v[w][q][lane];
+          for (int off = G; off < 32; off <<= 1) total[q] += __shfl_xor_sync(kAll, total[q], off);
+          if (grp == 0 && L.ok[q / VEC])
+            a.out[(size_t)u * a.F + L.base[q / VEC] + q % VEC] = total[q];
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
 // Forward: warp per destination row.  The indices of a row are read as coalesced batches of 32
 // (one per lane, the next batch in flight while the current one is used) and broadcast by
 // shuffles.  A lane holds four values of a message per edge: with VEC = 4 one 16-byte vector of
@@ -97,7 +384,8 @@ template <int BIN> struct EdgesInFlight {
 // vectors G apart, with VEC = 1 four features G apart; G lanes cover 4 G features per pass, and
 // vectors that lie beyond F are skipped for the whole warp.  Two or four edges per lane group are in flight per step.  No load is
 // predicated per lane: lanes without an edge or a feature read a valid address and their values
-// are dropped.
+// are dropped.  Rows longer than heavy_threshold are left to the leading blocks of the launch (see
+// fwd_heavy_rows) when a.heavy_list is set.
 template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a) {
   constexpr int kT = kTiles / VEC;  // vectors per lane and edge (4, 2 or 1)
@@ -105,11 +393,17 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
   // edges in flight per lane group and step: four where a message needs one vector load only
   constexpr int kEdges = (VEC > 1 && EdgesInFlight<BIN>::value == 4) ? 4 : 2;
   const int lane = threadIdx.x & 31;
-  const int64_t row = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
+  const int hb = a.heavy_list ? a.heavy_blocks : 0;
+  if ((int)blockIdx.x < hb) {
+    fwd_heavy_rows<BIN, RED, VEC>(a, blockIdx.x, hb);
+    return;
+  }
+  const int64_t row = (int64_t)(blockIdx.x - hb) * kGenWarps + (threadIdx.x >> 5);
   if (row >= a.n) return;
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
+  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this row
   const int F = a.F, cols = a.cols;
   for (int f0 = 0; f0 < F; f0 += kT * G * VEC) {
     bool ok[kT], tile_on[kT];
@@ -226,18 +520,25 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
 //   dV[u][j] = sum_q sel * dO[v_q][j] * d(x (x) y)/dx,   sel = [arg[v_q][j] == perm[q]] (max/min)
 // The derivative depends on y only (and not at all for copylhs / add / sub).  Same walk as the
 // forward kernel: batched indices (destination and CSR position), four values per lane and edge
-// in vectors of VEC floats, unpredicated loads.
+// in vectors of VEC floats, unpredicated loads; the handle's heavy columns go to the leading blocks
+// (bwd_heavy_cols).
 template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const GenArgs a) {
   constexpr int kT = kTiles / VEC;
   constexpr int NV = kT * VEC;
   constexpr int kEdges = 2;
   const int lane = threadIdx.x & 31;
-  const int64_t u = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
+  const int hb = a.heavy_list ? a.heavy_blocks : 0;
+  if ((int)blockIdx.x < hb) {
+    bwd_heavy_cols<BIN, RED, VEC>(a, blockIdx.x, hb);
+    return;
+  }
+  const int64_t u = (int64_t)(blockIdx.x - hb) * kGenWarps + (threadIdx.x >> 5);
   if (u >= a.n) return;
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   const int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
+  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this column
   const int F = a.F, cols = a.cols;
   constexpr bool kNeedsY = BIN == kMul || BIN == kDiv;
   constexpr bool kNeedsK = kNeedsY || RED != kSum;
@@ -589,9 +890,10 @@ dg_status_t dispatch_ops(int bin, int red, const GenArgs& a, cudaStream_t s) {
 template <int BIN, int RED>
 struct FwdLauncher {
   static dg_status_t run(const GenArgs& a, cudaStream_t s) {
-    if (a.vec == 4) general_fwd_kernel<BIN, RED, 4><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
-    else if (a.vec == 2) general_fwd_kernel<BIN, RED, 2><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
-    else general_fwd_kernel<BIN, RED, 1><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
+    if (a.vec == 4) general_fwd_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
+    else if (a.vec == 2) general_fwd_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
+    else general_fwd_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
     DG_CUDA(cudaGetLastError());
     count_launches(1);
     return DG_OK;
@@ -600,9 +902,10 @@ struct FwdLauncher {
 template <int BIN, int RED>
 struct BwdVertexLauncher {
   static dg_status_t run(const GenArgs& a, cudaStream_t s) {
-    if (a.vec == 4) general_bwd_vertex_kernel<BIN, RED, 4><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
-    else if (a.vec == 2) general_bwd_vertex_kernel<BIN, RED, 2><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
-    else general_bwd_vertex_kernel<BIN, RED, 1><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);
+    const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
+    if (a.vec == 4) general_bwd_vertex_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
+    else if (a.vec == 2) general_bwd_vertex_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
+    else general_bwd_vertex_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
     DG_CUDA(cudaGetLastError());
     count_launches(1);
     return DG_OK;
@@ -663,6 +966,13 @@ dg_status_t dg_ap_fwd(dg_graph_t g, const float* fV, const float* fE, int32_t fE
   if (binary != DG_BIN_COPY_LHS && a.cols != 1) both |= (uintptr_t)fE;
   a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
   a.log_g = log_group(F / a.vec);
+  if (g->nnz > g->heavy_threshold) {  // only then can a row be on the heavy list
+    a.heavy_list = g->heavy_rows;
+    a.heavy_count = g->counters + 0;
+    a.heavy_cap = (int32_t)g->heavy_cap;
+    a.heavy_threshold = (int32_t)g->heavy_threshold;
+    a.heavy_blocks = g->sm_count * 4;
+  }
   return dispatch_ops<FwdLauncher>((int)binary, (int)reduce, a, (cudaStream_t)stream);
 }
 
@@ -700,6 +1010,13 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
       if (reduce != DG_RED_SUM) both |= (uintptr_t)arg;
       a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
       a.log_g = log_group(F / a.vec);
+      if (g->nnz > g->heavy_threshold) {  // the heavy columns of the CSC
+        a.heavy_list = g->heavy_cols;
+        a.heavy_count = g->counters + 1;
+        a.heavy_cap = (int32_t)g->heavy_cap;
+        a.heavy_threshold = (int32_t)g->heavy_threshold;
+        a.heavy_blocks = g->sm_count * 4;
+      }
       if (dg_status_t st = dispatch_ops<BwdVertexLauncher>((int)binary, (int)reduce, a, s)) return st;
     }
   }

@@ -30,9 +30,11 @@ def edge_features(nnz, cols, seed, device=DEV):
     return torch.rand((nnz, cols), generator=gen, device=device, dtype=torch.float32) * 1.5 + 0.5
 
 
-def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False):
+def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False, heavy_threshold=None):
     g = make_graph(sg)
     g.dg_graph_transpose()
+    if heavy_threshold is not None:
+        g.dg_graph_set_param("heavy_threshold", heavy_threshold)
     rp, ci = to_np(sg.rowptr), to_np(sg.colidx)
     X = synth.features(sg.n, F, 500 + seed, DEV)
     Y = edge_features(sg.nnz, cols, 600 + seed)
@@ -94,6 +96,19 @@ def test_scaled_workloads(name, scale, F):
     sg = synth.make(name, device=DEV, scale=scale)
     for binary, reduce, cols in ((4, 0, F), (4, 0, 1), (0, 1, 1), (3, 2, F), (5, 0, F)):
         run_case(sg, F, cols, binary, reduce, seed=binary + reduce)
+
+
+@pytest.mark.parametrize("F,cols", [(64, 64), (100, 1), (7, 7), (260, 1)])
+def test_heavy_rows_and_columns_take_the_block_kernels(F, cols):
+    """With the lowest threshold most rows of the Reddit-like graph (and most columns of its
+    transpose) are on the handle's heavy lists, so the leading blocks of the launch compute them:
+    eight warps per row, merged in shared memory.  Sums within the bound, max / min and their
+    arg bit-exact with ties (few distinct values) going to the lowest edge position."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.01)
+    assert int((sg.rowptr[1:] - sg.rowptr[:-1]).max()) > 64 * 8   # rows of more than 8 batches
+    for binary, reduce, ties in ((0, 0, False), (4, 0, False), (0, 1, True), (2, 2, True),
+                                 (5, 0, False), (4, 1, False)):
+        run_case(sg, F, cols, binary, reduce, seed=F + binary, tie_heavy=ties, heavy_threshold=64)
 
 
 def test_empty_rows_and_empty_graph():
