@@ -275,6 +275,11 @@ dg_status_t dg_permute_rows(const int32_t* new_of_old, int64_t n, int32_t F, con
  * and among equal messages the one at the lowest edge position wins.  A message is one fp32
  * IEEE operation on the two fp32 operands, so the result of max / min is exact and the same on
  * every run; sums are fp32 in a fixed order.
+ * Where fV does not fit the handle's L2 budget and the rows are long and sorted, the call runs
+ * as one launch per (range of source ids, slice of 128 features) as the sum / mean calls do
+ * (attributes "l2_budget_mb", "source_blocks"); each launch folds its piece into fO, for max /
+ * min through arg, so a caller who passes arg = NULL gets feature slices only.  fO and arg must
+ * not overlap the inputs.
  * Asynchronous on `stream`.
  */
 typedef enum {

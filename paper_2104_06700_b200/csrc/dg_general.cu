@@ -52,6 +52,13 @@ struct GenArgs {
   const int32_t* heavy_count;
   int32_t heavy_cap, heavy_threshold;
   int32_t heavy_blocks;  // leading blocks of the grid that walk the heavy list
+  // one pass of a sliced / source-blocked call (forward and gradient with respect to fV):
+  // features [f_lo, f_lo + f_cnt), the piece [seg_lo[v], seg_hi[v]) of every row (nullptr: whole
+  // rows), and whether out (and arg_out) already hold the result of the earlier pieces
+  int32_t f_lo, f_cnt;
+  const int32_t* seg_lo;
+  const int32_t* seg_hi;
+  int32_t accumulate;
 };
 
 // one fp32 IEEE operation, never contracted into a neighbouring add
@@ -232,10 +239,12 @@ __device__ __forceinline__ void fwd_heavy_rows(const GenArgs& a, int first, int 
   const int count = min(*a.heavy_count, a.heavy_cap);
   for (int i = first; i < count; i += stride) {
     const int64_t row = a.heavy_list[i];
-    const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
-    for (int f0 = 0; f0 < a.F; f0 += kTiles * G) {
+    const int64_t lo = a.seg_lo ? __ldg(a.seg_lo + row) : __ldg(a.ptr + row);
+    const int64_t hi = a.seg_hi ? __ldg(a.seg_hi + row) : __ldg(a.ptr + row + 1);
+    const int f_end = a.f_lo + a.f_cnt;
+    for (int f0 = a.f_lo; f0 < f_end; f0 += kTiles * G) {
       LaneTiles<VEC> L;
-      L.place(f0, a.F, G, c);
+      L.place(f0, f_end, G, c);
       float total[4], best[4];
       int32_t best_k[4];
       fwd_walk<BIN, RED, VEC>(a, lo, hi, warp, kGenWarps, L, grp, NG, total, best, best_k);
@@ -265,8 +274,9 @@ __device__ __forceinline__ void fwd_heavy_rows(const GenArgs& a, int first, int 
           if (grp == 0 && L.ok[q / VEC]) {
             const size_t o = (size_t)row * a.F + L.base[q / VEC] + q % VEC;
             if (RED == kSum) {
-              a.out[o] = total[q];
+              a.out[o] = a.accumulate ? a.out[o] + total[q] : total[q];
             } else {
+              if (a.accumulate) take_better<RED>(best[q], best_k[q], a.out[o], a.arg_out[o]);
               a.out[o] = best_k[q] >= 0 ? best[q] : 0.f;
               if (a.arg_out) a.arg_out[o] = best_k[q];
             }
@@ -353,10 +363,12 @@ __device__ __forceinline__ void bwd_heavy_cols(const GenArgs& a, int first, int 
   const int count = min(*a.heavy_count, a.heavy_cap);
   for (int i = first; i < count; i += stride) {
     const int64_t u = a.heavy_list[i];
-    const int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
-    for (int f0 = 0; f0 < a.F; f0 += kTiles * G) {
+    const int64_t lo = a.seg_lo ? __ldg(a.seg_lo + u) : __ldg(a.ptr + u);
+    const int64_t hi = a.seg_hi ? __ldg(a.seg_hi + u) : __ldg(a.ptr + u + 1);
+    const int f_end = a.f_lo + a.f_cnt;
+    for (int f0 = a.f_lo; f0 < f_end; f0 += kTiles * G) {
       LaneTiles<VEC> L;
-      L.place(f0, a.F, G, c);
+      L.place(f0, f_end, G, c);
       float total[4];
       bwd_walk<BIN, RED, VEC>(a, lo, hi, warp, kGenWarps, L, grp, NG, total);
 #pragma unroll
@@ -368,8 +380,10 @@ __device__ __forceinline__ void bwd_heavy_cols(const GenArgs& a, int first, int 
           if (!L.tile_on[q / VEC]) continue;
           for (int w = 1; w < kGenWarps; ++w) total[q] += part_v[w][q][lane];
           for (int off = G; off < 32; off <<= 1) total[q] += __shfl_xor_sync(kAll, total[q], off);
-          if (grp == 0 && L.ok[q / VEC])
-            a.out[(size_t)u * a.F + L.base[q / VEC] + q % VEC] = total[q];
+          if (grp == 0 && L.ok[q / VEC]) {
+            float* o = a.out + (size_t)u * a.F + L.base[q / VEC] + q % VEC;
+            *o = a.accumulate ? *o + total[q] : total[q];
+          }
         }
       }
       __syncthreads();
@@ -402,18 +416,23 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
   if (row >= a.n) return;
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
-  const int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
+  int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
   if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this row
+  if (a.seg_lo) {  // this launch's piece of the row (one range of source ids)
+    lo = __ldg(a.seg_lo + row);
+    hi = __ldg(a.seg_hi + row);
+  }
   const int F = a.F, cols = a.cols;
-  for (int f0 = 0; f0 < F; f0 += kT * G * VEC) {
+  const int f_end = a.f_lo + a.f_cnt;
+  for (int f0 = a.f_lo; f0 < f_end; f0 += kT * G * VEC) {
     bool ok[kT], tile_on[kT];
     int base[kT];  // first feature of the lane's vector t (0 when it lies beyond F)
     float acc[NV], total[NV], best[NV];
     int32_t best_k[NV];
 #pragma unroll
     for (int t = 0; t < kT; ++t) {
-      tile_on[t] = f0 + t * G * VEC < F;             // the same for the whole warp
-      ok[t] = f0 + (t * G + c) * VEC < F;
+      tile_on[t] = f0 + t * G * VEC < f_end;         // the same for the whole warp
+      ok[t] = f0 + (t * G + c) * VEC < f_end;
       base[t] = ok[t] ? f0 + (t * G + c) * VEC : 0;
     }
 #pragma unroll
@@ -506,8 +525,9 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
       if (grp == 0 && ok[q / VEC]) {
         const size_t o = (size_t)row * F + base[q / VEC] + q % VEC;
         if (RED == kSum) {
-          a.out[o] = total[q];
+          a.out[o] = a.accumulate ? a.out[o] + total[q] : total[q];
         } else {
+          if (a.accumulate) take_better<RED>(best[q], best_k[q], a.out[o], a.arg_out[o]);
           a.out[o] = best_k[q] >= 0 ? best[q] : 0.f;
           if (a.arg_out) a.arg_out[o] = best_k[q];
         }
@@ -537,19 +557,24 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
   if (u >= a.n) return;
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
-  const int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
+  int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
   if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this column
+  if (a.seg_lo) {  // this launch's piece of the column (one range of destination ids)
+    lo = __ldg(a.seg_lo + u);
+    hi = __ldg(a.seg_hi + u);
+  }
   const int F = a.F, cols = a.cols;
+  const int f_end = a.f_lo + a.f_cnt;
   constexpr bool kNeedsY = BIN == kMul || BIN == kDiv;
   constexpr bool kNeedsK = kNeedsY || RED != kSum;
-  for (int f0 = 0; f0 < F; f0 += kT * G * VEC) {
+  for (int f0 = a.f_lo; f0 < f_end; f0 += kT * G * VEC) {
     bool ok[kT], tile_on[kT];
     int base[kT];
     float acc[NV], total[NV];
 #pragma unroll
     for (int t = 0; t < kT; ++t) {
-      tile_on[t] = f0 + t * G * VEC < F;
-      ok[t] = f0 + (t * G + c) * VEC < F;
+      tile_on[t] = f0 + t * G * VEC < f_end;
+      ok[t] = f0 + (t * G + c) * VEC < f_end;
       base[t] = ok[t] ? f0 + (t * G + c) * VEC : 0;
     }
 #pragma unroll
@@ -624,7 +649,10 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
       if (!tile_on[q / VEC]) continue;
       total[q] += acc[q];
       for (int off = G; off < 32; off <<= 1) total[q] += __shfl_xor_sync(kAll, total[q], off);
-      if (grp == 0 && ok[q / VEC]) a.out[(size_t)u * F + base[q / VEC] + q % VEC] = total[q];
+      if (grp == 0 && ok[q / VEC]) {
+        float* o = a.out + (size_t)u * F + base[q / VEC] + q % VEC;
+        *o = a.accumulate ? *o + total[q] : total[q];
+      }
     }
   }
 }
@@ -856,6 +884,39 @@ int log_group(int32_t width) {  // lanes per edge: the power of two covering `wi
   return lg;
 }
 
+// Feature slices and source blocks of one general call, like the sum / mean kernels' (Algorithm 2
+// with L2 as the cache): when the gathered matrices (`gathered` of them, n x F floats each) do not
+// fit the handle's L2 budget, the call runs as one launch per (range of neighbour ids, slice of 128
+// features: one walk of a row with 32 lanes x 4 values); the ranges partition the edges and each
+// launch folds its piece into the output of the earlier ones (can_merge: max / min need the arg
+// matrix for that).  Without split pointers, or where the pieces of a row would fall under 32
+// edges, slices alone are used if one slice of all rows fits; otherwise the call stays one launch.
+// The handle's "source_blocks" attribute forces the number of ranges.
+void plan_pieces(const dg_graph* g, int32_t F, int gathered, const int32_t* split, bool can_merge,
+                 int64_t* slice, int* nb) {
+  *slice = F;
+  *nb = 1;
+  const double budget = (double)g->l2_budget_bytes;
+  const int64_t w = F < 128 ? F : 128;
+  const double row_bytes = (double)(w * 4 + 128) * gathered;  // a slice rarely starts on a line
+  if (split && can_merge && g->source_blocks > 1) {
+    *slice = w;
+    *nb = (int)g->source_blocks;
+    return;
+  }
+  if (g->source_blocks == 1 || (double)g->n * F * 4.0 * gathered <= budget) return;
+  if (split && can_merge) {
+    int cand = 1;
+    while (cand < kFineBlocks && (double)g->n / cand * row_bytes > budget) cand *= 2;
+    if ((double)g->nnz / (double)g->n / cand >= 32.0) {
+      *slice = w;
+      *nb = cand;
+      return;
+    }
+  }
+  if ((double)g->n * row_bytes <= budget) *slice = w;
+}
+
 inline unsigned warp_blocks(int64_t n) { return (unsigned)((n + kGenWarps - 1) / kGenWarps); }
 
 template <template <int, int> class L>
@@ -911,6 +972,25 @@ struct BwdVertexLauncher {
     return DG_OK;
   }
 };
+// one launch per piece; L::run launches the kernel of the operator pair
+template <template <int, int> class L>
+dg_status_t run_pieces(const dg_graph* g, GenArgs a, int bin, int red, const int32_t* split,
+                       int64_t slice, int nb, cudaStream_t s) {
+  const int per = kFineBlocks / nb;
+  for (int j = 0; j < nb; ++j) {
+    if (nb > 1) {
+      a.seg_lo = split + (size_t)(j * per) * (size_t)g->n;
+      a.seg_hi = split + (size_t)((j + 1) * per) * (size_t)g->n;
+    }
+    a.accumulate = j > 0;
+    for (int64_t f0 = 0; f0 < a.F; f0 += slice) {
+      a.f_lo = (int32_t)f0;
+      a.f_cnt = (int32_t)(a.F - f0 < slice ? a.F - f0 : slice);
+      if (dg_status_t st = dispatch_ops<L>(bin, red, a, s)) return st;
+    }
+  }
+  return DG_OK;
+}
 DG_GEN_LAUNCHER(BwdEdgeFullLauncher, general_bwd_edge_full_kernel)
 DG_GEN_LAUNCHER(BwdEdgeScalarLauncher, general_bwd_edge_scalar_kernel)
 #undef DG_GEN_LAUNCHER
@@ -973,7 +1053,13 @@ dg_status_t dg_ap_fwd(dg_graph_t g, const float* fV, const float* fE, int32_t fE
     a.heavy_threshold = (int32_t)g->heavy_threshold;
     a.heavy_blocks = g->sm_count * 4;
   }
-  return dispatch_ops<FwdLauncher>((int)binary, (int)reduce, a, (cudaStream_t)stream);
+  int64_t slice;
+  int nb;
+  // copyrhs gathers nothing: its edge rows are a stream
+  plan_pieces(g, F, binary == DG_BIN_COPY_RHS ? 0 : 1, g->split_csr,
+              reduce == DG_RED_SUM || arg != nullptr, &slice, &nb);
+  return run_pieces<FwdLauncher>(g, a, (int)binary, (int)reduce, g->split_csr, slice, nb,
+                                 (cudaStream_t)stream);
 }
 
 dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const float* fE,
@@ -1017,7 +1103,12 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
         a.heavy_threshold = (int32_t)g->heavy_threshold;
         a.heavy_blocks = g->sm_count * 4;
       }
-      if (dg_status_t st = dispatch_ops<BwdVertexLauncher>((int)binary, (int)reduce, a, s)) return st;
+      int64_t slice;
+      int nb;
+      plan_pieces(g, F, reduce == DG_RED_SUM ? 1 : 2, g->split_csc, true, &slice, &nb);  // dO, arg
+      if (dg_status_t st = run_pieces<BwdVertexLauncher>(g, a, (int)binary, (int)reduce,
+                                                         g->split_csc, slice, nb, s))
+        return st;
     }
   }
   if (dE && g->nnz > 0) {

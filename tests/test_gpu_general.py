@@ -30,11 +30,14 @@ def edge_features(nnz, cols, seed, device=DEV):
     return torch.rand((nnz, cols), generator=gen, device=device, dtype=torch.float32) * 1.5 + 0.5
 
 
-def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False, heavy_threshold=None):
+def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False, heavy_threshold=None,
+             params=None, min_launches=0):
     g = make_graph(sg)
     g.dg_graph_transpose()
     if heavy_threshold is not None:
         g.dg_graph_set_param("heavy_threshold", heavy_threshold)
+    for name, value in (params or {}).items():
+        g.dg_graph_set_param(name, value)
     rp, ci = to_np(sg.rowptr), to_np(sg.colidx)
     X = synth.features(sg.n, F, 500 + seed, DEV)
     Y = edge_features(sg.nnz, cols, 600 + seed)
@@ -44,8 +47,10 @@ def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False, heavy_thresho
     G = synth.features(sg.n, F, 700 + seed, DEV)
     fV = None if binary == binding.DG_BIN_COPY_RHS else X
     fE = None if binary == binding.DG_BIN_COPY_LHS else Y
+    before = binding.dg_kernel_launch_count()
     out, arg = g.dg_ap_fwd(fV, fE, binary, reduce, F=F)
     torch.cuda.synchronize()
+    assert binding.dg_kernel_launch_count() - before >= min_launches
     ref, mag, oarg = oracle.general_forward(rp, ci, to_np(fV), to_np(fE), binary, reduce, F=F)
     if reduce == binding.DG_RED_SUM:
         assert arg is None
@@ -53,8 +58,11 @@ def run_case(sg, F, cols, binary, reduce, seed=0, tie_heavy=False, heavy_thresho
     else:
         assert np.array_equal(to_np(out).astype(np.float64), ref), f"fwd {NAMES[binary]} max/min"
         assert np.array_equal(to_np(arg).astype(np.int64), oarg), "arg"
+    before = binding.dg_kernel_launch_count()
     dV, dE = g.dg_ap_bwd(G, fV, fE, binary, reduce, arg=arg)
     torch.cuda.synchronize()
+    if binary != binding.DG_BIN_COPY_RHS and "source_blocks" in (params or {}):
+        assert binding.dg_kernel_launch_count() - before >= min_launches
     odV, omV, odE, omE = oracle.general_backward(rp, ci, to_np(fV), to_np(fE), binary, reduce,
                                                  oarg, to_np(G))
     assert_within_bound(to_np(dV), odV, omV, f"dV {NAMES[binary]}")
@@ -109,6 +117,35 @@ def test_heavy_rows_and_columns_take_the_block_kernels(F, cols):
     for binary, reduce, ties in ((0, 0, False), (4, 0, False), (0, 1, True), (2, 2, True),
                                  (5, 0, False), (4, 1, False)):
         run_case(sg, F, cols, binary, reduce, seed=F + binary, tie_heavy=ties, heavy_threshold=64)
+
+
+@pytest.mark.parametrize("params,launches", [({"source_blocks": 4}, 8), ({"l2_budget_mb": 12}, 4),
+                                             ({"source_blocks": 16, "heavy_threshold": 64}, 32)])
+def test_feature_slices_and_source_blocks(params, launches):
+    """Cut into slices of 128 features and ranges of neighbour ids, one launch per piece, every
+    launch folding its piece into the output of the earlier ones: the same sums within the bound,
+    the same extrema and arg (bit-exact, ties to the lowest edge position) as in one launch."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.02)     # 32,946 vertices, 70 edges each
+    F = 196                                                    # slices of 128 and 68
+    for binary, reduce, cols, ties in ((4, 0, F, False), (0, 1, 1, True), (2, 2, F, True)):
+        run_case(sg, F, cols, binary, reduce, seed=31 + binary, tie_heavy=ties, params=params,
+                 min_launches=launches)
+
+
+def test_extrema_without_arg_are_not_cut_into_source_blocks():
+    """Folding a piece into the earlier ones needs the arg matrix; a caller that does not want it
+    still gets the right extrema."""
+    sg = synth.make("reddit_like", device=DEV, scale=0.02)
+    g = make_graph(sg)
+    g.dg_graph_set_param("source_blocks", 4)
+    F = 130
+    X = synth.features(sg.n, F, 77, DEV)
+    out, arg = g.dg_ap_fwd(X, None, binding.DG_BIN_COPY_LHS, binding.DG_RED_MAX, want_arg=False)
+    torch.cuda.synchronize()
+    assert arg is None
+    ref, _, _ = oracle.general_forward(to_np(sg.rowptr), to_np(sg.colidx), to_np(X), None,
+                                       binding.DG_BIN_COPY_LHS, binding.DG_RED_MAX, F=F)
+    assert np.array_equal(to_np(out).astype(np.float64), ref)
 
 
 def test_empty_rows_and_empty_graph():
