@@ -657,31 +657,50 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
   }
 }
 
-// Gradient with respect to fE, full edge features (cols == F): one value per (edge, feature),
+// Gradient with respect to fE: the output is per edge, so a row splits freely.  As in the
+// edge-weight gradient below, the first heavy_blocks blocks of a launch walk the handle's heavy
+// rows, the 8 warps of a block taking interleaved steps of one row (first = warp, stride = 8); in
+// the other blocks a warp owns one light row (first = 0, stride = 1).
+template <class Row>
+__device__ __forceinline__ void edge_rows(const GenArgs& a, Row row) {
+  const int warp = threadIdx.x >> 5;
+  const int hb = a.heavy_list ? a.heavy_blocks : 0;
+  if ((int)blockIdx.x < hb) {
+    const int count = min(*a.heavy_count, a.heavy_cap);
+    for (int i = blockIdx.x; i < count; i += hb) row(a.heavy_list[i], warp, kGenWarps);
+    return;
+  }
+  const int64_t v = (int64_t)(blockIdx.x - hb) * kGenWarps + warp;
+  if (v >= a.n) return;
+  if (a.heavy_list && __ldg(a.ptr + v + 1) - __ldg(a.ptr + v) > a.heavy_threshold) return;
+  row(v, 0, 1);
+}
+
+// Full edge features (cols == F): one value per (edge, feature),
 //   dE[k][j] = sel * dO[v][j] * d(x (x) y)/dy
 template <int BIN, int RED>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_full_kernel(const GenArgs a) {
-  const int lane = threadIdx.x & 31;
-  const int64_t v = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
-  if (v >= a.n) return;
-  const int G = 1 << a.log_g, NG = 32 >> a.log_g;
-  const int grp = lane >> a.log_g, c = lane & (G - 1);
-  const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
-  const int F = a.F;
-  constexpr bool kNeedsX = BIN == kMul || BIN == kDiv;
-  for (int f0 = 0; f0 < F; f0 += G) {
-    if (f0 + c >= F) continue;
-    const int j = f0 + c;
-    const float g = __ldg(a.X + (size_t)v * F + j);
-    const int32_t sel = RED != kSum ? __ldg(a.arg + (size_t)v * F + j) : 0;
-    for (int64_t e = lo + grp; e < hi; e += NG) {
-      const float x = kNeedsX ? __ldg(a.V + (size_t)__ldg(a.idx + e) * F + j) : 0.f;
-      const float y = BIN == kDiv ? __ldg(a.Y + (size_t)e * F + j) : 0.f;
-      float t = g * d_dy<BIN>(x, y);
-      if (RED != kSum && sel != (int32_t)e) t = 0.f;
-      a.out[(size_t)e * F + j] = t;
+  edge_rows(a, [&](int64_t v, int first, int stride) {
+    const int lane = threadIdx.x & 31;
+    const int G = 1 << a.log_g, NG = 32 >> a.log_g;
+    const int grp = lane >> a.log_g, c = lane & (G - 1);
+    const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
+    const int F = a.F;
+    constexpr bool kNeedsX = BIN == kMul || BIN == kDiv;
+    for (int f0 = 0; f0 < F; f0 += G) {
+      if (f0 + c >= F) continue;
+      const int j = f0 + c;
+      const float g = __ldg(a.X + (size_t)v * F + j);
+      const int32_t sel = RED != kSum ? __ldg(a.arg + (size_t)v * F + j) : 0;
+      for (int64_t e = lo + (int64_t)first * NG + grp; e < hi; e += (int64_t)stride * NG) {
+        const float x = kNeedsX ? __ldg(a.V + (size_t)__ldg(a.idx + e) * F + j) : 0.f;
+        const float y = BIN == kDiv ? __ldg(a.Y + (size_t)e * F + j) : 0.f;
+        float t = g * d_dy<BIN>(x, y);
+        if (RED != kSum && sel != (int32_t)e) t = 0.f;
+        a.out[(size_t)e * F + j] = t;
+      }
     }
-  }
+  });
 }
 
 // Gradient with respect to fE with one column (the broadcast scalar): the feature sum of the
@@ -691,32 +710,33 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_full_kernel(const 
 // gradient with respect to a scalar edge weight; row_scale gives the mean's s_v.
 template <int BIN, int RED>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_scalar_kernel(const GenArgs a) {
-  const int lane = threadIdx.x & 31;
-  const int64_t v = (int64_t)blockIdx.x * kGenWarps + (threadIdx.x >> 5);
-  if (v >= a.n) return;
-  const int G = 1 << a.log_g, NG = 32 >> a.log_g;
-  const int grp = lane >> a.log_g, c = lane & (G - 1);
-  const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
-  const int F = a.F;
-  constexpr bool kNeedsX = BIN == kMul || BIN == kDiv;
-  float s = 1.f;
-  if (a.row_scale) s = 1.0f / (float)(hi - lo + (a.row_scale == 2 ? 1 : 0));
-  for (int64_t e0 = lo; e0 < hi; e0 += NG) {   // uniform trip count: the shuffles need all lanes
-    const int64_t e = e0 + grp;
-    const bool eok = e < hi;
-    float dot = 0.f;
-    if (eok) {
-      const float* xrow = kNeedsX ? a.V + (size_t)__ldg(a.idx + e) * F : nullptr;
-      const float y = BIN == kDiv ? __ldg(a.Y + e) : 0.f;
-      for (int j = c; j < F; j += G) {
-        float t = __ldg(a.X + (size_t)v * F + j) * d_dy<BIN>(kNeedsX ? __ldg(xrow + j) : 0.f, y);
-        if (RED != kSum && __ldg(a.arg + (size_t)v * F + j) != (int32_t)e) t = 0.f;
-        dot += t;
+  edge_rows(a, [&](int64_t v, int first, int stride) {
+    const int lane = threadIdx.x & 31;
+    const int G = 1 << a.log_g, NG = 32 >> a.log_g;
+    const int grp = lane >> a.log_g, c = lane & (G - 1);
+    const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
+    const int F = a.F;
+    constexpr bool kNeedsX = BIN == kMul || BIN == kDiv;
+    float s = 1.f;
+    if (a.row_scale) s = 1.0f / (float)(hi - lo + (a.row_scale == 2 ? 1 : 0));
+    // uniform trip count per warp: the shuffles need all lanes
+    for (int64_t e0 = lo + (int64_t)first * NG; e0 < hi; e0 += (int64_t)stride * NG) {
+      const int64_t e = e0 + grp;
+      const bool eok = e < hi;
+      float dot = 0.f;
+      if (eok) {
+        const float* xrow = kNeedsX ? a.V + (size_t)__ldg(a.idx + e) * F : nullptr;
+        const float y = BIN == kDiv ? __ldg(a.Y + e) : 0.f;
+        for (int j = c; j < F; j += G) {
+          float t = __ldg(a.X + (size_t)v * F + j) * d_dy<BIN>(kNeedsX ? __ldg(xrow + j) : 0.f, y);
+          if (RED != kSum && __ldg(a.arg + (size_t)v * F + j) != (int32_t)e) t = 0.f;
+          dot += t;
+        }
       }
+      for (int off = 1; off < G; off <<= 1) dot += __shfl_xor_sync(kAll, dot, off);
+      if (eok && c == 0) a.out[e] = dot * s;
     }
-    for (int off = 1; off < G; off <<= 1) dot += __shfl_xor_sync(kAll, dot, off);
-    if (eok && c == 0) a.out[e] = dot * s;
-  }
+  });
 }
 
 // ---- dg_aggregate_edge_grad: dW[k] = s_v * <H[u_k], dOut[v_k]>, one dot product per edge ----
@@ -942,7 +962,8 @@ dg_status_t dispatch_ops(int bin, int red, const GenArgs& a, cudaStream_t s) {
   template <int BIN, int RED>                                                 \
   struct NAME {                                                               \
     static dg_status_t run(const GenArgs& a, cudaStream_t s) {                \
-      KERNEL<BIN, RED><<<warp_blocks(a.n), kGenBlock, 0, s>>>(a);             \
+      const unsigned heavy = a.heavy_list ? (unsigned)a.heavy_blocks : 0u;    \
+      KERNEL<BIN, RED><<<heavy + warp_blocks(a.n), kGenBlock, 0, s>>>(a);     \
       DG_CUDA(cudaGetLastError());                                            \
       count_launches(1);                                                      \
       return DG_OK;                                                           \
@@ -1124,6 +1145,13 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
     a.F = F;
     a.cols = cols;
     a.log_g = log_group(F);
+    if (g->nnz > g->heavy_threshold) {
+      a.heavy_list = g->heavy_rows;
+      a.heavy_count = g->counters + 0;
+      a.heavy_cap = (int32_t)g->heavy_cap;
+      a.heavy_threshold = (int32_t)g->heavy_threshold;
+      a.heavy_blocks = g->sm_count * 4;
+    }
     if (cols == 1)
       return dispatch_ops<BwdEdgeScalarLauncher>((int)binary, (int)reduce, a, s);
     return dispatch_ops<BwdEdgeFullLauncher>((int)binary, (int)reduce, a, s);
