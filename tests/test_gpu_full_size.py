@@ -281,3 +281,113 @@ def test_full_size_products_like_hub_first():
         assert_within_bound(to_np(out), ref, mag, "fwd, hub-first")
         ref, mag = oracle.ap_backward(rp, colptr, rowidx_T, None, to_np(G), op)
         assert_within_bound(to_np(dH), ref, mag, "bwd, hub-first")
+
+
+def _row_sub_problem(ptr, idx, rows):
+    """The CSR rows `rows` as a graph of their own for the oracle: row i of the sub-problem is
+    rows[i], its sources are renumbered into `uniq`, and `pos` gives the position of every
+    sub-problem edge in the full arrays.  Padded with empty rows so that row and source ids
+    share one range."""
+    sp, si, _, uniq, pos = sample_segments(ptr, idx, None, rows)
+    n_sub = max(len(rows), uniq.numel())
+    return _pad_ptr(sp, n_sub), si, uniq, pos, n_sub
+
+
+def _column_sub_problem(g, cols):
+    """The out-edges of the source vertices `cols` as a CSR graph of their own: its rows are the
+    destinations they reach (`dests`, renumbered), its sources are 0..len(cols)-1, the edges of
+    a row keep their CSR order, and `k_full` gives the CSR position of every edge in the full
+    graph (ascending, because CSR positions grow with the row)."""
+    colptr, rowidx_T, _, perm = g.dg_graph_get_csc()
+    sp, si, _, dests, posT = sample_segments(colptr, rowidx_T, None, cols)
+    owner = np.repeat(np.arange(len(cols), dtype=np.int32), np.diff(sp))
+    k_full = to_np(perm[posT]).astype(np.int64)
+    order = np.argsort(k_full, kind="stable")          # CSR order = (row, position in row)
+    k_full, dest_sub, src_sub = k_full[order], si[order], owner[order]
+    assert np.all(np.diff(dest_sub) >= 0)
+    n_sub = max(len(cols), dests.numel())
+    rp = np.zeros(n_sub + 1, dtype=np.int64)
+    np.add.at(rp, dest_sub.astype(np.int64) + 1, 1)
+    return np.cumsum(rp), src_sub, dests, k_full, n_sub
+
+
+@pytest.mark.parametrize("name,F,fE_cols", [("reddit_like", 602, 1), ("products_like", 100, 1),
+                                            ("proteins_like", 64, 64)])
+def test_full_size_general_calls(name, F, fE_cols):
+    """dg_ap_fwd / dg_ap_bwd (copylhs / max with arg, mul / sum with edge features) and
+    dg_aggregate_edge_grad at full size with default knobs, i.e. in the launch shapes the
+    benchmark times: feature slices x source blocks on the Reddit-like graph, block-per-row heavy
+    rows and columns on the Products-like one, the full |E| x F edge-feature stream on the
+    Proteins-like one.  Every output row (edge) depends on its own CSR row (CSC column) only, so
+    the oracle computes sampled rows and columns as sub-problems: random ones plus the longest,
+    which take the block-per-row path.  The extrema and their arg are compared bit for bit; the
+    vertex gradient of max is also checked through the identity that every non-empty (v, j)
+    hands its dO to exactly one source: sum_u dV[u][j] = sum_{v: arg >= 0} dO[v][j]."""
+    sg = synth.make(name, device=DEV)
+    g = binding.dg_graph_create(sg.n, sg.nnz, sg.rowptr, sg.colidx, None)
+    g.dg_graph_validate()
+    g.dg_graph_transpose()
+    colptr = g.dg_graph_get_csc()[0]
+    H = synth.features(sg.n, F, 61, DEV)
+    G = synth.features(sg.n, F, 62, DEV)
+    rows = pick_rows(sg.rowptr, sg.n, 150, 12, 63)
+    cols = pick_rows(colptr, sg.n, 60, 3, 64)
+    ridx, cidx = torch.as_tensor(rows, device=DEV), torch.as_tensor(cols, device=DEV)
+    rp_r, ci_r, uniq_r, pos_r, n_r = _row_sub_problem(sg.rowptr, sg.colidx, rows)
+    rp_c, ci_c, dests_c, k_c, n_c = _column_sub_problem(g, cols)
+    H_r = _pad_rows(to_np(H[uniq_r]), n_r)
+    G_r = _pad_rows(to_np(G[ridx]), n_r)
+    G_c = _pad_rows(to_np(G[dests_c]), n_c)
+    H_c = _pad_rows(to_np(H[cidx]), n_c)
+    k = len(rows)
+    assert k >= 150 and pos_r.numel() > 1000 and len(k_c) > 1000    # real sub-problems
+
+    # -- copylhs / max: extrema and arg bit-exact on the sampled rows
+    out, arg = g.dg_ap_fwd(H, None, binding.DG_BIN_COPY_LHS, binding.DG_RED_MAX)
+    torch.cuda.synchronize()
+    ref, _, oarg = oracle.general_forward(rp_r, ci_r, H_r, None, binding.DG_BIN_COPY_LHS,
+                                          binding.DG_RED_MAX)
+    assert np.array_equal(to_np(out[ridx]).astype(np.float64), ref[:k]), "max"
+    pos_np = to_np(pos_r).astype(np.int64)
+    want_arg = np.where(oarg[:k] >= 0, pos_np[np.maximum(oarg[:k], 0)], -1)
+    assert np.array_equal(to_np(arg[ridx]).astype(np.int64), want_arg), "arg"
+    assert (want_arg >= 0).mean() > 0.5
+    # -- its vertex gradient on the sampled columns, given that arg
+    dV, _ = g.dg_ap_bwd(G, H, None, binding.DG_BIN_COPY_LHS, binding.DG_RED_MAX, arg=arg)
+    torch.cuda.synchronize()
+    arg_c = to_np(arg[dests_c]).astype(np.int64)             # full positions -> sub positions
+    at = np.minimum(np.searchsorted(k_c, arg_c), len(k_c) - 1)
+    arg_sub = np.full((n_c, F), -1, dtype=np.int64)
+    arg_sub[:arg_c.shape[0]] = np.where(k_c[at] == arg_c, at, -1)
+    assert (arg_sub >= 0).any()                      # some extrema do come from the sampled sources
+    odV, omV, _, _ = oracle.general_backward(rp_c, ci_c, H_c, None, binding.DG_BIN_COPY_LHS,
+                                             binding.DG_RED_MAX, arg_sub, G_c)
+    assert_within_bound(to_np(dV[cidx]), odV[:len(cols)], omV[:len(cols)], "dV of max")
+    routed = torch.where(arg >= 0, G, torch.zeros_like(G)).double()
+    total, scale = routed.sum(0), routed.abs().sum(0)
+    assert bool(((dV.double().sum(0) - total).abs() <= 1e-5 * scale + 1e-7).all()), "sum of dV"
+    del out, arg, dV, routed
+
+    # -- mul / sum with edge features: forward, dV and dE
+    fE = torch.rand((sg.nnz, fE_cols), device=DEV, dtype=torch.float32) + 0.5
+    out, _ = g.dg_ap_fwd(H, fE, binding.DG_BIN_MUL, binding.DG_RED_SUM)
+    dV, dE = g.dg_ap_bwd(G, H, fE, binding.DG_BIN_MUL, binding.DG_RED_SUM)
+    torch.cuda.synchronize()
+    fE_r = to_np(fE[pos_r])
+    ref, mag, _ = oracle.general_forward(rp_r, ci_r, H_r, fE_r, binding.DG_BIN_MUL,
+                                         binding.DG_RED_SUM)
+    assert_within_bound(to_np(out[ridx]), ref[:k], mag[:k], "mul/sum")
+    _, _, odE, omE = oracle.general_backward(rp_r, ci_r, H_r, fE_r, binding.DG_BIN_MUL,
+                                             binding.DG_RED_SUM, None, G_r, want_dV=False)
+    assert_within_bound(to_np(dE[pos_r]), odE, omE, "dE of mul/sum")
+    fE_c = to_np(fE[torch.as_tensor(k_c, device=DEV)])
+    odV, omV, _, _ = oracle.general_backward(rp_c, ci_c, H_c, fE_c, binding.DG_BIN_MUL,
+                                             binding.DG_RED_SUM, None, G_c, want_dE=False)
+    assert_within_bound(to_np(dV[cidx]), odV[:len(cols)], omV[:len(cols)], "dV of mul/sum")
+    del out, dV, dE, fE
+
+    # -- gradient with respect to scalar edge weights of the mean
+    dW = g.dg_aggregate_edge_grad(H, G, binding.DG_OP_MEAN)
+    torch.cuda.synchronize()
+    ref, mag = oracle.edge_weight_grad(rp_r, ci_r, H_r, G_r, binding.DG_OP_MEAN)
+    assert_within_bound(to_np(dW[pos_r]), ref, mag, "dW")
