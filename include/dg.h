@@ -279,7 +279,8 @@ dg_status_t dg_permute_rows(const int32_t* new_of_old, int64_t n, int32_t F, con
  * as one launch per (range of source ids, slice of 128 features) as the sum / mean calls do
  * (attributes "l2_budget_mb", "source_blocks"); each launch folds its piece into fO, for max /
  * min through arg, so a caller who passes arg = NULL gets feature slices only.  fO and arg must
- * not overlap the inputs.
+ * not overlap the inputs.  copylhs / sum and mul / sum with fE_cols = 1 are the plain and the
+ * weighted sum: these two pairs run on the kernels of dg_aggregate_fwd (fE as the weights).
  * Asynchronous on `stream`.
  */
 typedef enum {

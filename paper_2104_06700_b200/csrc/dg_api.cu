@@ -210,6 +210,30 @@ static dg_status_t run_backward(Graph* g, const void* dOut, bool bf16, int32_t F
   return aggregate_run(g, a, sa, g->split_csc, (cudaStream_t)stream);
 }
 
+// sum_k w_k X[idx[k]] over the CSR rows (or the CSC columns) with the sum / mean kernels, for
+// the operator pairs of the general entry points that are exactly this.  w is in the order of
+// the direction walked, or nullptr; the handle's own weights and its "self_loops" attribute play
+// no part.
+dg_status_t aggregate_sum(Graph* g, bool over_csc, const float* w, const float* X, int32_t F,
+                          float* Y, cudaStream_t s) {
+  ApArgs a{};
+  a.ptr = over_csc ? g->colptr : g->rowptr;
+  a.idx = over_csc ? g->rowidx_T : g->colidx;
+  a.w = w;
+  a.X = X;
+  a.Y = Y;
+  a.heavy_list = over_csc ? g->heavy_cols : g->heavy_rows;
+  a.heavy_count = g->counters + (over_csc ? 1 : 0);
+  a.heavy_cap = (int32_t)g->heavy_cap;
+  a.n = g->n;
+  a.F = F;
+  a.heavy_threshold = (int32_t)g->heavy_threshold;
+  a.rows_per_warp = rows_per_warp(g);
+  a.long_segments = over_csc ? long_columns(g) : g->long_rows;
+  a.full_registers = full_registers(g);
+  return aggregate_run(g, a, SelfArgs{nullptr, 0}, over_csc ? g->split_csc : g->split_csr, s);
+}
+
 static dg_status_t malformed(int flags) {
   set_error("malformed CSR:%s%s%s%s", (flags & 1) ? " rowptr[0] != 0;" : "",
             (flags & 2) ? " rowptr decreases;" : "", (flags & 4) ? " rowptr[n] != nnz;" : "",

@@ -972,25 +972,36 @@ dg_status_t dispatch_ops(int bin, int red, const GenArgs& a, cudaStream_t s) {
 template <int BIN, int RED>
 struct FwdLauncher {
   static dg_status_t run(const GenArgs& a, cudaStream_t s) {
-    const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
-    if (a.vec == 4) general_fwd_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
-    else if (a.vec == 2) general_fwd_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
-    else general_fwd_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
-    DG_CUDA(cudaGetLastError());
-    count_launches(1);
-    return DG_OK;
+    if constexpr (BIN == kCopyLhs && RED == kSum) {  // dg_ap_fwd hands this pair to aggregate_sum
+      (void)a; (void)s;
+      return DG_ERR_UNSUPPORTED;
+    } else {
+      const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
+      if (a.vec == 4) general_fwd_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
+      else if (a.vec == 2) general_fwd_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
+      else general_fwd_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
+      DG_CUDA(cudaGetLastError());
+      count_launches(1);
+      return DG_OK;
+    }
   }
 };
 template <int BIN, int RED>
 struct BwdVertexLauncher {
   static dg_status_t run(const GenArgs& a, cudaStream_t s) {
-    const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
-    if (a.vec == 4) general_bwd_vertex_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
-    else if (a.vec == 2) general_bwd_vertex_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
-    else general_bwd_vertex_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
-    DG_CUDA(cudaGetLastError());
-    count_launches(1);
-    return DG_OK;
+    // dg_ap_bwd hands the pairs whose derivative is 1 to aggregate_sum
+    if constexpr (RED == kSum && (BIN == kCopyLhs || BIN == kAdd || BIN == kSub)) {
+      (void)a; (void)s;
+      return DG_ERR_UNSUPPORTED;
+    } else {
+      const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
+      if (a.vec == 4) general_bwd_vertex_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
+      else if (a.vec == 2) general_bwd_vertex_kernel<BIN, RED, 2><<<grid, kGenBlock, 0, s>>>(a);
+      else general_bwd_vertex_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
+      DG_CUDA(cudaGetLastError());
+      count_launches(1);
+      return DG_OK;
+    }
   }
 };
 // one launch per piece; L::run launches the kernel of the operator pair
@@ -1052,6 +1063,12 @@ dg_status_t dg_ap_fwd(dg_graph_t g, const float* fV, const float* fE, int32_t fE
   if (dg_status_t st = check_operands(g, fV, fE, fE_cols, F, (int)binary, (int)reduce)) return st;
   if (g->n == 0) return DG_OK;
   if (!fO) return bad("fO is NULL");
+  // copylhs / sum is the plain sum, mul / sum with one column the weighted sum with fE as the
+  // weights: the sum / mean kernels do these two (about 2.5x faster on the dense graphs)
+  if (reduce == DG_RED_SUM &&
+      (binary == DG_BIN_COPY_LHS || (binary == DG_BIN_MUL && fE_cols == 1)))
+    return aggregate_sum(g, false, binary == DG_BIN_MUL ? fE : nullptr, fV, F, fO,
+                         (cudaStream_t)stream);
   GenArgs a{};
   a.ptr = g->rowptr;
   a.idx = g->colidx;
@@ -1101,35 +1118,41 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
         set_error("the gradient with respect to fV gathers over the CSC: call dg_graph_transpose first");
         return DG_ERR_NOT_TRANSPOSED;
       }
-      GenArgs a{};
-      a.ptr = g->colptr;
-      a.idx = g->rowidx_T;
-      a.perm = g->perm;
-      a.X = dO;
-      a.Y = fE;
-      a.arg = arg;
-      a.out = dV;
-      a.n = g->n;
-      a.F = F;
-      a.cols = cols;
-      uintptr_t both = (uintptr_t)dO;
-      if ((binary == DG_BIN_MUL || binary == DG_BIN_DIV) && cols != 1) both |= (uintptr_t)fE;
-      if (reduce != DG_RED_SUM) both |= (uintptr_t)arg;
-      a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
-      a.log_g = log_group(F / a.vec);
-      if (g->nnz > g->heavy_threshold) {  // the heavy columns of the CSC
-        a.heavy_list = g->heavy_cols;
-        a.heavy_count = g->counters + 1;
-        a.heavy_cap = (int32_t)g->heavy_cap;
-        a.heavy_threshold = (int32_t)g->heavy_threshold;
-        a.heavy_blocks = g->sm_count * 4;
+      // sum with copylhs / add / sub: dV[u] is the plain sum of dO over the out-edges of u
+      if (reduce == DG_RED_SUM && (binary == DG_BIN_COPY_LHS || binary == DG_BIN_ADD ||
+                                   binary == DG_BIN_SUB)) {
+        if (dg_status_t st = aggregate_sum(g, true, nullptr, dO, F, dV, s)) return st;
+      } else {
+        GenArgs a{};
+        a.ptr = g->colptr;
+        a.idx = g->rowidx_T;
+        a.perm = g->perm;
+        a.X = dO;
+        a.Y = fE;
+        a.arg = arg;
+        a.out = dV;
+        a.n = g->n;
+        a.F = F;
+        a.cols = cols;
+        uintptr_t both = (uintptr_t)dO;
+        if ((binary == DG_BIN_MUL || binary == DG_BIN_DIV) && cols != 1) both |= (uintptr_t)fE;
+        if (reduce != DG_RED_SUM) both |= (uintptr_t)arg;
+        a.vec = (F % 4 == 0 && (both & 15) == 0) ? 4 : (F % 2 == 0 && (both & 7) == 0) ? 2 : 1;
+        a.log_g = log_group(F / a.vec);
+        if (g->nnz > g->heavy_threshold) {  // the heavy columns of the CSC
+          a.heavy_list = g->heavy_cols;
+          a.heavy_count = g->counters + 1;
+          a.heavy_cap = (int32_t)g->heavy_cap;
+          a.heavy_threshold = (int32_t)g->heavy_threshold;
+          a.heavy_blocks = g->sm_count * 4;
+        }
+        int64_t slice;
+        int nb;
+        plan_pieces(g, F, reduce == DG_RED_SUM ? 1 : 2, g->split_csc, true, &slice, &nb);  // dO, arg
+        if (dg_status_t st = run_pieces<BwdVertexLauncher>(g, a, (int)binary, (int)reduce,
+                                                           g->split_csc, slice, nb, s))
+          return st;
       }
-      int64_t slice;
-      int nb;
-      plan_pieces(g, F, reduce == DG_RED_SUM ? 1 : 2, g->split_csc, true, &slice, &nb);  // dO, arg
-      if (dg_status_t st = run_pieces<BwdVertexLauncher>(g, a, (int)binary, (int)reduce,
-                                                         g->split_csc, slice, nb, s))
-        return st;
     }
   }
   if (dE && g->nnz > 0) {

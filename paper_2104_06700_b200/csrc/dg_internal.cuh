@@ -166,5 +166,9 @@ dg_status_t expand_rows(const int64_t* rowptr, int64_t n, int64_t nnz, const int
 // dg_aggregate.cu
 dg_status_t aggregate_run(const Graph* g, const ApArgs& a, const SelfArgs& sa, const int32_t* split,
                           cudaStream_t s);
+// sum_k w_k X[idx[k]] over the CSR rows or the CSC columns with those kernels (dg_api.cu); w in
+// the order of that direction or nullptr, no self loops.
+dg_status_t aggregate_sum(Graph* g, bool over_csc, const float* w, const float* X, int32_t F,
+                          float* Y, cudaStream_t s);
 
 }  // namespace dg
