@@ -105,10 +105,11 @@ def parse_args():
                          "contiguous) instead of a random permutation; reported separately")
     ap.add_argument("--reorder", default="none", choices=["none", "out_degree", "in_degree"],
                     help="rename the vertices hub-first with dg_graph_reorder before the run "
-                         "(reported separately; combine with --set hub_rows=N for the hub pass)")
+                         "(reported separately)")
     ap.add_argument("--other-calls", action="store_true",
                     help="also time dg_aggregate_edge_grad and two dg_ap_fwd operator pairs on "
-                         "the chosen workload (the default run does so on two workloads)")
+                         "the chosen workload (the default run does so on the headline workload "
+                         "and on two others)")
     ap.add_argument("--workloads", default="all", choices=["all", "none"],
                     help="all: after the headline step, one record per workload shape at full "
                          "size (default run on one GPU only); none: the headline alone")
@@ -1092,14 +1093,15 @@ def main():
 
     # ---------------------------------------------------------------- every workload shape (N = 1)
     workloads = workloads_ingest = workloads_epoch = workloads_extras = None
-    if rank == 0 and world == 1 and args.other_calls and not two_buffers:
+    default_run = (args.workload == "reddit_like" and args.scale == 1.0 and not args.feat
+                   and not bf16 and not args.set and not args.sorted_ids and op == "mean"
+                   and args.reorder == "none")
+    want_extras = args.other_calls or (default_run and args.workloads == "all")
+    if rank == 0 and world == 1 and want_extras and not two_buffers:
         flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
         workloads_extras = extra_records(torch, binding, synth, args.workload, g, sg, F, n_ref, peak,
                                          flush_buf)
         del flush_buf
-    default_run = (args.workload == "reddit_like" and args.scale == 1.0 and not args.feat
-                   and not bf16 and not args.set and not args.sorted_ids and op == "mean"
-                   and args.reorder == "none")
     if rank == 0 and world == 1 and args.workloads == "all" and default_run:
         head = {"workload": args.workload, "scale": 1.0, "n": sg.n, "nnz": sg.nnz, "F": F, "op": op,
                 "weighted": weighted, "reorder": "none", "dtype": "f32", "reps": args.steps,
@@ -1114,11 +1116,13 @@ def main():
                        "transpose_edges_per_s": sg.nnz / (transpose_ms * 1e-3)}
         del H, out, G, dH, g, csc, sg
         torch.cuda.empty_cache()
+        head_extras = workloads_extras or []
         workloads, workloads_ingest, workloads_epoch, workloads_extras = run_workloads(
             torch, binding, synth, dev, local_rank, peak, ceilings,
             0.0 if args.no_cpu_baseline else min(3.0, args.cpu_seconds),
             skip={(args.workload, F, op)})
         workloads.insert(2, head)
+        workloads_extras = head_extras + workloads_extras
         workloads_ingest[args.workload + " (headline run)"] = ingest_head
         sg = type("Shape", (), {"n": head["n"], "nnz": head["nnz"]})()
 
