@@ -313,7 +313,7 @@ def probe_rate(binding, torch, dev, table_bytes, row_floats, count=1 << 25, reps
 
 def run_probe():
     """Random-row gather rates of this GPU (one JSON line): from an L2-resident and an HBM-sized
-    table (dg_probe_gather), and from a block's own and a cluster partner's shared memory
+    table and from a mix of the two (dg_probe_gather), and from a block's own and a cluster partner's shared memory
     (dg_probe_gather_smem), each also as bytes per clock per SM at the SM clock sampled meanwhile."""
     import torch
     from paper_2104_06700_b200 import binding
@@ -358,6 +358,21 @@ def run_probe():
                   row_floats * 4)
             del table, idx
             torch.cuda.empty_cache()
+    # mixed traffic: a share of the gathers goes to a hot set that stays in L2, the rest anywhere in
+    # an HBM-sized table (what a power-law graph does to the forward pass)
+    rows, hot_rows = int(16e9 // 512), int(30e6 // 512)
+    table = torch.zeros((rows, 128), dtype=torch.float32, device=dev)
+    for share in (0.25, 0.5, 0.75):
+        idx = torch.randint(0, rows, (count,), generator=gen, device=dev, dtype=torch.int32)
+        hot = torch.randint(0, hot_rows, (count,), generator=gen, device=dev, dtype=torch.int32)
+        pick = torch.rand(count, generator=gen, device=dev) < share
+        idx = torch.where(pick, hot * (rows // hot_rows), idx)
+        del hot, pick
+        timed(lambda: binding.dg_probe_gather(table, idx, sink),
+              f"mixed_hbm_16GB_hot_30MB_share{int(share * 100)}_row512B", 512)
+        del idx
+    del table
+    torch.cuda.empty_cache()
     for remote in (False, True):
         for row_floats in (128, 32, 16, 8):
             stage_rows = (192 * 1024) // (row_floats * 4)
