@@ -302,8 +302,13 @@ constexpr size_t scatter_smem_bytes() {
 
 // colptr[u] = first position q whose sorted key is >= u.  Position q fills the ids between the
 // key before it and its own key; position nnz closes the array up to n.  A thread takes
-// kColptrItems consecutive positions (one 16-byte load when `vector_ok`: sorted 16-byte aligned).
+// kColptrItems consecutive positions (one 16-byte load when `vector_ok`: sorted 16-byte aligned)
+// and fills at most the last kMaxFill ids of a gap itself: a long run of ids without a key (a
+// hub-first numbering puts every vertex without out-edges at the end, millions of them) would
+// otherwise be one thread's loop (Papers-like x0.1, hub-first: 17 ms).  The ids it leaves keep
+// the -1 the array was filled with, and fill_long_gaps finds each by a binary search.
 constexpr int kColptrItems = 4;
+constexpr int kMaxFill = 32;
 __global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int64_t nnz,
                                         int64_t n, int vector_ok, int64_t* __restrict__ colptr) {
   const int64_t q0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * kColptrItems;
@@ -324,9 +329,25 @@ __global__ void colptr_from_sorted_keys(const uint32_t* __restrict__ sorted, int
     int64_t cur = q < nnz ? (int64_t)k[i] : n;
     const int64_t next_prev = cur;
     if (cur > n) cur = n;  // an id outside [0, n) must not turn into a write outside colptr
-    for (int64_t u = prev + 1; u <= cur; ++u) colptr[u] = q;
+    int64_t u = prev + 1;
+    if (cur - u >= kMaxFill) u = cur - kMaxFill + 1;
+    for (; u <= cur; ++u) colptr[u] = q;
     prev = next_prev;
   }
+}
+
+// the ids colptr_from_sorted_keys left at -1: the first position whose key is >= u, by search
+__global__ void fill_long_gaps(const uint32_t* __restrict__ sorted, int64_t nnz, int64_t n,
+                               int64_t* __restrict__ colptr) {
+  const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (u > n || colptr[u] >= 0) return;
+  int64_t lo = 0, hi = nnz;  // invariant: keys before lo are < u, keys from hi on are >= u
+  while (lo < hi) {
+    const int64_t mid = (lo + hi) >> 1;
+    if ((int64_t)__ldg(sorted + mid) < u) lo = mid + 1;
+    else hi = mid;
+  }
+  colptr[u] = lo;
 }
 
 // row_info[k] = (row r with rowptr[r] <= k < rowptr[r+1], bits of 1/(deg(r) + self)) for every
@@ -562,10 +583,13 @@ dg_status_t sort_pairs(const uint32_t* keys_in, const uint32_t* vals_in, int64_t
 // ptr[u] = first position whose sorted key is >= u, for u = 0..n (ptr[n] = count)
 dg_status_t pointers_from_sorted_keys(const uint32_t* sorted, int64_t count, int64_t n,
                                       int64_t* ptr, cudaStream_t s) {
+  DG_CUDA(cudaMemsetAsync(ptr, 0xFF, (size_t)(n + 1) * sizeof(int64_t), s));  // -1 everywhere
   const unsigned blocks = (unsigned)(((count + kColptrItems) / kColptrItems + 255) / 256);
   colptr_from_sorted_keys<<<blocks, 256, 0, s>>>(sorted, count, n, aligned16(sorted), ptr);
   DG_CUDA(cudaGetLastError());
-  count_launches(1);
+  fill_long_gaps<<<(unsigned)((n + 1 + 255) / 256), 256, 0, s>>>(sorted, count, n, ptr);
+  DG_CUDA(cudaGetLastError());
+  count_launches(2);
   return DG_OK;
 }
 
