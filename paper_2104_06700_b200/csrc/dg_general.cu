@@ -13,9 +13,9 @@
 // bytes, read once, coalesced), so these passes are bound by HBM streaming rather than by the
 // gather.
 //
-// Determinism: every output element is produced by one warp (one block) in a fixed order; the extremum of
-// max / min is chosen on (message, edge position) pairs, equal messages going to the lowest
-// position, so the order in which lane groups are combined does not matter.  No atomics.
+// Determinism: every output element is produced by one warp (one block) in a fixed order; the
+// extremum of max / min is chosen on (message, edge position) pairs, equal messages going to the
+// lowest position, so the order in which lane groups are combined does not matter.  No atomics.
 #include "dg_internal.cuh"
 
 namespace dg {
@@ -396,10 +396,10 @@ __device__ __forceinline__ void bwd_heavy_cols(const GenArgs& a, int first, int 
 // shuffles.  A lane holds four values of a message per edge: with VEC = 4 one 16-byte vector of
 // consecutive features (F a multiple of 4, 16-byte aligned matrices), with VEC = 2 two 8-byte
 // vectors G apart, with VEC = 1 four features G apart; G lanes cover 4 G features per pass, and
-// vectors that lie beyond F are skipped for the whole warp.  Two or four edges per lane group are in flight per step.  No load is
-// predicated per lane: lanes without an edge or a feature read a valid address and their values
-// are dropped.  Rows longer than heavy_threshold are left to the leading blocks of the launch (see
-// fwd_heavy_rows) when a.heavy_list is set.
+// vectors that lie beyond F are skipped for the whole warp.  Two or four edges per lane group are
+// in flight per step.  No load is predicated per lane: lanes without an edge or a feature read a
+// valid address and their values are dropped.  Rows longer than heavy_threshold are left to the
+// leading blocks of the launch (see fwd_heavy_rows) when a.heavy_list is set.
 template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a) {
   constexpr int kT = kTiles / VEC;  // vectors per lane and edge (4, 2 or 1)
@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   int64_t lo = __ldg(a.ptr + row), hi = __ldg(a.ptr + row + 1);
-  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this row
+  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk has it
   if (a.seg_lo) {  // this launch's piece of the row (one range of source ids)
     lo = __ldg(a.seg_lo + row);
     hi = __ldg(a.seg_hi + row);
@@ -558,7 +558,7 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_vertex_kernel(const Gen
   const int G = 1 << a.log_g, NG = 32 >> a.log_g;
   const int grp = lane >> a.log_g, c = lane & (G - 1);
   int64_t lo = __ldg(a.ptr + u), hi = __ldg(a.ptr + u + 1);
-  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk writes this column
+  if (a.heavy_list && hi - lo > a.heavy_threshold) return;  // a block of the list walk has it
   if (a.seg_lo) {  // this launch's piece of the column (one range of destination ids)
     lo = __ldg(a.seg_lo + u);
     hi = __ldg(a.seg_hi + u);
