@@ -590,7 +590,15 @@ def extra_records(torch, binding, synth, name, g, sg, F, n_ref, peak, flush):
         out.append(rec("dg_ap_fwd (mul, sum), |E| x F edge features", ms,
                        idx_bytes + n_ref * F * 4 + sg.n * F * 4 + sg.nnz * F * 4,
                        "the edge stream (nnz x F x 4 bytes, read once) dominates: HBM-streaming bound"))
-        del fE
+        dE = torch.empty_like(fE)
+        bwd_e = lambda: binding._check(binding.lib().dg_ap_bwd(
+            g._h, G.data_ptr(), H.data_ptr(), fE.data_ptr(), F, F, binding.DG_BIN_MUL,
+            binding.DG_RED_SUM, None, None, dE.data_ptr(), torch.cuda.current_stream().cuda_stream))
+        ms = time_one(torch, bwd_e, 10, None)
+        out.append(rec("dg_ap_bwd (mul, sum): dE, |E| x F", ms,
+                       idx_bytes + n_ref * F * 4 + sg.n * F * 4 + sg.nnz * F * 4,
+                       "dE[k] = dO[v] * fV[u]: one written row per edge (nnz x F x 4 bytes) dominates"))
+        del fE, dE
     return out
 
 

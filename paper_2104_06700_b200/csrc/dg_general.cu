@@ -678,7 +678,9 @@ __device__ __forceinline__ void edge_rows(const GenArgs& a, Row row) {
 
 // Full edge features (cols == F): one value per (edge, feature),
 //   dE[k][j] = sel * dO[v][j] * d(x (x) y)/dy
-template <int BIN, int RED>
+// G lanes per edge, VEC consecutive features per lane (16-byte loads and stores when F is a
+// multiple of 4 and the matrices are 16-byte aligned): the written rows are the traffic.
+template <int BIN, int RED, int VEC>
 __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_full_kernel(const GenArgs a) {
   edge_rows(a, [&](int64_t v, int first, int stride) {
     const int lane = threadIdx.x & 31;
@@ -687,17 +689,26 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_full_kernel(const 
     const int64_t lo = __ldg(a.ptr + v), hi = __ldg(a.ptr + v + 1);
     const int F = a.F;
     constexpr bool kNeedsX = BIN == kMul || BIN == kDiv;
-    for (int f0 = 0; f0 < F; f0 += G) {
-      if (f0 + c >= F) continue;
-      const int j = f0 + c;
-      const float g = __ldg(a.X + (size_t)v * F + j);
-      const int32_t sel = RED != kSum ? __ldg(a.arg + (size_t)v * F + j) : 0;
+    for (int f0 = 0; f0 < F; f0 += G * VEC) {
+      const int j = f0 + c * VEC;
+      if (j >= F) continue;
+      float g[VEC], x[VEC], y[VEC], t[VEC];
+      int32_t sel[VEC];
+      load_vec<VEC>(g, a.X + (size_t)v * F + j);
+#pragma unroll
+      for (int q = 0; q < VEC; ++q) { sel[q] = 0; x[q] = y[q] = 0.f; }
+      if (RED != kSum) load_vec<VEC>(sel, a.arg + (size_t)v * F + j);
       for (int64_t e = lo + (int64_t)first * NG + grp; e < hi; e += (int64_t)stride * NG) {
-        const float x = kNeedsX ? __ldg(a.V + (size_t)__ldg(a.idx + e) * F + j) : 0.f;
-        const float y = BIN == kDiv ? __ldg(a.Y + (size_t)e * F + j) : 0.f;
-        float t = g * d_dy<BIN>(x, y);
-        if (RED != kSum && sel != (int32_t)e) t = 0.f;
-        a.out[(size_t)e * F + j] = t;
+        if (kNeedsX) load_vec<VEC>(x, a.V + (size_t)__ldg(a.idx + e) * F + j);
+        if (BIN == kDiv) load_vec<VEC>(y, a.Y + (size_t)e * F + j);
+#pragma unroll
+        for (int q = 0; q < VEC; ++q) {
+          t[q] = g[q] * d_dy<BIN>(x[q], y[q]);
+          if (RED != kSum && sel[q] != (int32_t)e) t[q] = 0.f;
+        }
+        float* o = a.out + (size_t)e * F + j;
+        if (VEC == 4) *reinterpret_cast<float4*>(o) = make_float4(t[0], t[1], t[2], t[3]);
+        else o[0] = t[0];
       }
     }
   });
@@ -1023,7 +1034,17 @@ dg_status_t run_pieces(const dg_graph* g, GenArgs a, int bin, int red, const int
   }
   return DG_OK;
 }
-DG_GEN_LAUNCHER(BwdEdgeFullLauncher, general_bwd_edge_full_kernel)
+template <int BIN, int RED>
+struct BwdEdgeFullLauncher {
+  static dg_status_t run(const GenArgs& a, cudaStream_t s) {
+    const unsigned grid = (a.heavy_list ? (unsigned)a.heavy_blocks : 0u) + warp_blocks(a.n);
+    if (a.vec == 4) general_bwd_edge_full_kernel<BIN, RED, 4><<<grid, kGenBlock, 0, s>>>(a);
+    else general_bwd_edge_full_kernel<BIN, RED, 1><<<grid, kGenBlock, 0, s>>>(a);
+    DG_CUDA(cudaGetLastError());
+    count_launches(1);
+    return DG_OK;
+  }
+};
 DG_GEN_LAUNCHER(BwdEdgeScalarLauncher, general_bwd_edge_scalar_kernel)
 #undef DG_GEN_LAUNCHER
 
@@ -1167,7 +1188,15 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
     a.n = g->n;
     a.F = F;
     a.cols = cols;
-    a.log_g = log_group(F);
+    a.vec = 1;
+    if (cols != 1) {  // 16-byte rows of every matrix the full-width kernel touches
+      uintptr_t all = (uintptr_t)dO | (uintptr_t)dE;
+      if (binary == DG_BIN_MUL || binary == DG_BIN_DIV) all |= (uintptr_t)fV;
+      if (binary == DG_BIN_DIV) all |= (uintptr_t)fE;
+      if (reduce != DG_RED_SUM) all |= (uintptr_t)arg;
+      if (F % 4 == 0 && (all & 15) == 0) a.vec = 4;
+    }
+    a.log_g = log_group(F / a.vec);
     if (g->nnz > g->heavy_threshold) {
       a.heavy_list = g->heavy_rows;
       a.heavy_count = g->counters + 0;
