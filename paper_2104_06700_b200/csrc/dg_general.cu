@@ -101,7 +101,7 @@ __device__ __forceinline__ void take_better(float& best, int32_t& best_k, float 
 constexpr int kTiles = 4;  // feature tiles of G lanes a warp carries through one walk of a row
 // edges in flight per lane group and step: four where only one operand is loaded per message
 template <int BIN> struct EdgesInFlight {
-  static constexpr int value = (BIN == kCopyLhs || BIN == kCopyRhs) ? 4 : 2;
+  static constexpr int value = 4;
 };
 
 // ---- rows on the handle's heavy list: a block per row ----
@@ -463,21 +463,21 @@ __global__ void __launch_bounds__(kGenBlock) general_fwd_kernel(const GenArgs a)
               float2 xv = make_float2(0.f, 0.f), yv = make_float2(y1, y1);
               if (BIN != kCopyRhs) xv = __ldg(reinterpret_cast<const float2*>(xrow + base[t]));
               if (BIN != kCopyLhs && cols != 1)
-                yv = __ldg(reinterpret_cast<const float2*>(yrow + base[t]));
+                yv = __ldcs(reinterpret_cast<const float2*>(yrow + base[t]));
               x[i][t * 2 + 0] = xv.x; x[i][t * 2 + 1] = xv.y;
               y[i][t * 2 + 0] = yv.x; y[i][t * 2 + 1] = yv.y;
             } else if (VEC == 4) {
               float4 xv = make_float4(0.f, 0.f, 0.f, 0.f), yv = make_float4(y1, y1, y1, y1);
               if (BIN != kCopyRhs) xv = __ldg(reinterpret_cast<const float4*>(xrow + base[t]));
               if (BIN != kCopyLhs && cols != 1)
-                yv = __ldg(reinterpret_cast<const float4*>(yrow + base[t]));
+                yv = __ldcs(reinterpret_cast<const float4*>(yrow + base[t]));
               x[i][t * 4 + 0] = xv.x; x[i][t * 4 + 1] = xv.y;
               x[i][t * 4 + 2] = xv.z; x[i][t * 4 + 3] = xv.w;
               y[i][t * 4 + 0] = yv.x; y[i][t * 4 + 1] = yv.y;
               y[i][t * 4 + 2] = yv.z; y[i][t * 4 + 3] = yv.w;
             } else {
               x[i][t] = BIN != kCopyRhs ? __ldg(xrow + base[t]) : 0.f;
-              y[i][t] = (BIN != kCopyLhs && cols != 1) ? __ldg(yrow + base[t]) : y1;
+              y[i][t] = (BIN != kCopyLhs && cols != 1) ? __ldcs(yrow + base[t]) : y1;
             }
           }
         }
@@ -707,8 +707,9 @@ __global__ void __launch_bounds__(kGenBlock) general_bwd_edge_full_kernel(const 
           if (RED != kSum && sel[q] != (int32_t)e) t[q] = 0.f;
         }
         float* o = a.out + (size_t)e * F + j;
-        if (VEC == 4) *reinterpret_cast<float4*>(o) = make_float4(t[0], t[1], t[2], t[3]);
-        else o[0] = t[0];
+        // written once, never read here: streaming stores leave L2 to the gathered rows
+        if (VEC == 4) __stcs(reinterpret_cast<float4*>(o), make_float4(t[0], t[1], t[2], t[3]));
+        else __stcs(o, t[0]);
       }
     }
   });
