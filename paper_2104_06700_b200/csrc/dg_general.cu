@@ -1178,6 +1178,9 @@ dg_status_t dg_ap_bwd(dg_graph_t g, const float* dO, const float* fV, const floa
     }
   }
   if (dE && g->nnz > 0) {
+    // mul / sum with one edge column: dE[k] = <fV[u_k], dO[v_k]>, the edge-weight gradient of the sum
+    if (binary == DG_BIN_MUL && reduce == DG_RED_SUM && cols == 1)
+      return dg_aggregate_edge_grad(g, fV, dO, F, DG_OP_SUM, dE, stream);
     GenArgs a{};
     a.ptr = g->rowptr;
     a.idx = g->colidx;
