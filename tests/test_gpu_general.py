@@ -126,7 +126,7 @@ def test_feature_slices_and_source_blocks(params, launches):
     launch folding its piece into the output of the earlier ones: the same sums within the bound,
     the same extrema and arg (bit-exact, ties to the lowest edge position) as in one launch."""
     sg = synth.make("reddit_like", device=DEV, scale=0.02)     # 32,946 vertices, 70 edges each
-    F = 196                                                    # slices of 128 and 68
+    F = 132                                                    # slices of 128 and 4
     for binary, reduce, cols, ties in ((4, 0, F, False), (0, 1, 1, True), (2, 2, F, True)):
         run_case(sg, F, cols, binary, reduce, seed=31 + binary, tie_heavy=ties, params=params,
                  min_launches=launches)
